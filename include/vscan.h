@@ -1,0 +1,222 @@
+/*
+ * vscan.h - C ABI of the VScan visual-token reduction library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the two reduction points of VScan:
+ *   Stage 1 (Sec. 4.1), at the vision-encoder output, per encoder instance (image or crop):
+ *     vscan_score (ROW mode)        head mean of the [CLS] attention rows          (Eq. 1-2)
+ *     vscan_select_global_local     per-window top-k + global top-k, union         (Eq. 2-3)
+ *     vscan_merge                   cosine arg-max assignment + mean merge         (Eq. 4)
+ *   Stage 2 (Sec. 4.2), at a middle LLM layer, per sequence:
+ *     vscan_score (QK mode)         head mean of softmax(q_last . K) over a span   (Eq. 5)
+ *     vscan_llm_prune               that score + top-k + compaction of hidden / K / V / position ids
+ *
+ * Conventions shared by every entry point
+ *   - Returns a vscan_status.  Nothing throws, aborts or traps.  Arguments are validated on the
+ *     host before any launch; on a validation error nothing is enqueued.
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller, contiguous (row-major) in the
+ *     layout stated, at least 16-byte aligned.  Inputs are only read.  Outputs must not overlap
+ *     inputs.  NULL is allowed only where "optional" is written.
+ *   - The library allocates no device memory and keeps no state between calls.  Scratch memory is
+ *     a caller-provided `workspace` of at least vscan_*_workspace_bytes(desc) bytes, 256-byte
+ *     aligned; its contents before the call are irrelevant and after the call unspecified.
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     is asynchronous with respect to the host; no call synchronises.
+ *   - `dtype` is the element type of features, attention rows, q, K, V and hidden states
+ *     (VSCAN_F32 or VSCAN_BF16).  Scores are always float32, indices int32.
+ *   - Ties: wherever a top-k or an arg-max meets equal values the lowest index wins.  Survivor
+ *     lists are in ascending original index.
+ *   - Shapes are uniform over the batch of one call.  Counts (k_global, k_per_window, k_keep) are
+ *     explicit integers; percentages (R1, R2 of the paper) are resolved by the caller.
+ */
+#ifndef VSCAN_H_
+#define VSCAN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VSCAN_VERSION 100 /* major*10000 + minor*100 + patch */
+
+typedef enum {
+  VSCAN_OK = 0,
+  VSCAN_ERR_INVALID_ARG = 1, /* null pointer, bad range, misalignment, overlap */
+  VSCAN_ERR_UNSUPPORTED = 2, /* legal request this build cannot run (shape limit, dtype/path) */
+  VSCAN_ERR_WORKSPACE = 3,   /* workspace missing, misaligned or too small */
+  VSCAN_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, no sm_100 device) */
+  VSCAN_ERR_TIMEOUT = 5      /* a bounded device-side wait ran out (reported by vscan_check) */
+} vscan_status;
+
+typedef enum { VSCAN_F32 = 0, VSCAN_BF16 = 1 } vscan_dtype;
+typedef enum { VSCAN_SCORE_ROW = 0, VSCAN_SCORE_QK = 1 } vscan_score_mode;
+/* Eq. 5 takes the softmax over the visual keys only (SPAN_ONLY); Sec. 4.2's remark on recomputing
+ * "vanilla attention" for the last token normalises over all keys (SPAN_FULL). */
+typedef enum { VSCAN_SPAN_ONLY = 0, VSCAN_SPAN_FULL = 1 } vscan_softmax_span;
+/* Which unit runs the similarity contraction of vscan_merge. */
+typedef enum {
+  VSCAN_MERGE_AUTO = 0,   /* tensor cores for bf16 when the shape allows, else CUDA cores */
+  VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
+  VSCAN_MERGE_TENSOR = 2  /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory */
+} vscan_merge_path;
+
+/* ---------------------------------------------------------------------------------------------
+ * vscan_score
+ *
+ * ROW mode (Eq. 2): scores[b][j] = (1/heads) * sum_h attn[b][h][cls_offset + j], j in [0, n_tokens).
+ *   attn      [instances][heads][row_len] of `dtype`: per-head attention probabilities of the [CLS]
+ *             query (Eq. 1) or, for encoders without [CLS] (text after Eq. 2), the per-head attention
+ *             each token receives, cls_offset = 0.  row_len >= cls_offset + n_tokens.
+ *             The skipped entries are ignored; the row is not renormalised.
+ *   scores    [instances][n_tokens] float32 (output).
+ * QK mode (Eq. 5): for each query head h with KV head g = floor(h * kv_heads / q_heads),
+ *   p_h = softmax_j(scale * q[b][h] . k[b][g][j]) taken over the span (SPAN_ONLY) or over all seq_len
+ *   keys (SPAN_FULL); scores[b][j] = (1/q_heads) * sum_h p_h[span_begin + j], j in [0, span_len).
+ *   q         [batch][q_heads][head_dim] of `dtype` (query of the last instruction token)
+ *   k         [batch][kv_heads][seq_len][head_dim] of `dtype`
+ *   scores    [batch][span_len] float32 (output).  head_dim must be a multiple of 8, at most 256;
+ *             q_heads a multiple of kv_heads.
+ * Fields of the mode not in use are ignored.  Workspace: QK mode only.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t mode;  /* vscan_score_mode */
+  int32_t dtype; /* vscan_dtype */
+  /* ROW */
+  const void* attn;
+  int32_t instances, heads, row_len, cls_offset, n_tokens;
+  /* QK */
+  const void* q;
+  const void* k;
+  int32_t batch, q_heads, kv_heads, seq_len, head_dim, span_begin, span_len;
+  int32_t softmax_span; /* vscan_softmax_span */
+  float scale;
+  /* output */
+  float* scores;
+} vscan_score_desc;
+
+size_t vscan_score_workspace_bytes(const vscan_score_desc* desc);
+vscan_status vscan_score(const vscan_score_desc* desc, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * vscan_select_global_local (Sec. 4.1, Eq. 2-3 and the footnote on duplicates)
+ *
+ * Tokens of an instance are numbered t = f*grid_h*grid_w + r*grid_w + c.  The grid is cut into
+ * non-overlapping win_h x win_w windows (win_h | grid_h, win_w | grid_w).
+ *   local scan : in every window the k_per_window tokens with the largest scores_local;
+ *   global scan: the k_global largest scores_global among the tokens the local scan did not take;
+ *   kept_idx   : the union, ascending, exactly K1 = windows*k_per_window + k_global per instance.
+ *   scores_global, scores_local  [instances][N] float32, N = frames*grid_h*grid_w (may be the same
+ *                                buffer)
+ *   kept_idx   [instances][K1] int32 (output)
+ *   kept_mask  [instances][N] uint8, 1 = kept (optional output)
+ * Legal ranges: 0 <= k_per_window <= win_h*win_w, 0 <= k_global <= N - windows*k_per_window.
+ * Limit of this build: N <= 16384.  No workspace needed (0 bytes).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  const float* scores_global;
+  const float* scores_local;
+  int32_t instances, frames, grid_h, grid_w, win_h, win_w, k_per_window, k_global;
+  int32_t* kept_idx;
+  uint8_t* kept_mask;
+} vscan_select_desc;
+
+size_t vscan_select_workspace_bytes(const vscan_select_desc* desc);
+vscan_status vscan_select_global_local(const vscan_select_desc* desc, void* workspace,
+                                       size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * vscan_merge (Sec. 4.1 "Token Merging", Eq. 4)
+ *
+ * For every token u not in kept_idx: a(u) = argmax_s cos(m_u, m_kept[s]) (lowest slot on ties; norms
+ * clamped at 1e-12), where m is `metric` if given, else x.  Then
+ *   merged[b][s] = (x_kept[s] + sum_{a(u)=s} x_u) / (1 + |{u : a(u)=s}|),
+ * accumulated in float32 in ascending token order and rounded once to `dtype`.
+ *   x         [instances][row_len][dim] of `dtype`; row cls_offset + t is token t; rows before
+ *             cls_offset (the [CLS] feature) are never read.  row_len >= cls_offset + n_tokens.
+ *   metric    optional [instances][row_len][metric_dim] of `dtype`
+ *   kept_idx  [instances][n_kept] int32, strictly ascending, each in [0, n_tokens)  (not checked
+ *             on the host; out-of-range entries are clamped on the device)
+ *   merged    [instances][n_kept][dim] of `dtype` (output)
+ *   assign    optional [instances][n_tokens] int32 output: slot of every token (a kept token maps
+ *             to its own slot).  When NULL it lives in the workspace.
+ *   counts    optional [instances][n_kept] int32 output: group size including the kept token.
+ * dim and metric_dim must be multiples of 8; 1 <= n_kept <= n_tokens.
+ * `path` picks the unit for the similarity contraction (vscan_merge_path).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t dtype; /* vscan_dtype */
+  int32_t path;  /* vscan_merge_path */
+  const void* x;
+  const void* metric;
+  const int32_t* kept_idx;
+  int32_t instances, row_len, cls_offset, n_tokens, dim, metric_dim, n_kept;
+  void* merged;
+  int32_t* assign;
+  int32_t* counts;
+} vscan_merge_desc;
+
+size_t vscan_merge_workspace_bytes(const vscan_merge_desc* desc);
+vscan_status vscan_merge(const vscan_merge_desc* desc, void* workspace, size_t workspace_bytes,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * vscan_llm_prune (Sec. 4.2; KV-cache remark of the same section)
+ *
+ * The sequence is [n_sys system | n_vis visual | n_txt text] tokens, seq_len = n_sys+n_vis+n_txt.
+ * Scores the visual span as vscan_score QK mode does (span_begin = n_sys, span_len = n_vis), keeps
+ * the k_keep highest, and writes the shortened sequence of seq_out = seq_len - n_vis + k_keep rows:
+ * system rows, surviving visual rows in ascending order, text rows.  Copies are bit-exact; position
+ * ids keep their original values.
+ *   q_last    [batch][q_heads][head_dim]           k, v   [batch][kv_heads][seq_len][head_dim]
+ *   hidden    [batch][seq_len][hidden_dim]         pos_ids [pos_planes][batch][seq_len] int32
+ *   kept_vis  [batch][k_keep] int32 output, indices relative to the visual span, ascending
+ *   hidden_out [batch][seq_out][hidden_dim]        k_out, v_out [batch][kv_heads][seq_out][head_dim]
+ *   pos_out   [pos_planes][batch][seq_out] int32
+ *   scores    optional [batch][n_vis] float32 output
+ * v/v_out, hidden/hidden_out and pos_ids/pos_out are optional as pairs (both NULL = skip).
+ * hidden_dim*sizeof(dtype) and head_dim*sizeof(dtype) must be multiples of 16.  0 <= k_keep <= n_vis.
+ * Limit of this build: n_vis <= 16384.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t dtype; /* vscan_dtype */
+  const void* q_last;
+  const void* k;
+  const void* v;
+  const void* hidden;
+  const int32_t* pos_ids;
+  int32_t batch, q_heads, kv_heads, head_dim, hidden_dim, pos_planes;
+  int32_t n_sys, n_vis, n_txt, k_keep;
+  int32_t softmax_span; /* vscan_softmax_span */
+  float scale;
+  int32_t* kept_vis;
+  void* hidden_out;
+  void* k_out;
+  void* v_out;
+  int32_t* pos_out;
+  float* scores;
+} vscan_prune_desc;
+
+size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* desc);
+vscan_status vscan_llm_prune(const vscan_prune_desc* desc, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Housekeeping.
+ * vscan_check: synchronises `stream` and reads the device status word at the start of a workspace
+ * that the preceding call used; VSCAN_OK, VSCAN_ERR_TIMEOUT (a bounded wait expired) or
+ * VSCAN_ERR_CUDA.  Only calls that take a non-empty workspace write that word.
+ * vscan_last_cuda_error: cudaError_t value of the last failing runtime call on this thread (0 if none).
+ * vscan_kernel_launches: number of kernels this library has launched in this process so far.
+ * ------------------------------------------------------------------------------------------- */
+int32_t vscan_version(void);
+const char* vscan_status_string(vscan_status status);
+vscan_status vscan_check(const void* workspace, void* stream);
+int32_t vscan_last_cuda_error(void);
+uint64_t vscan_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VSCAN_H_ */

@@ -1,0 +1,261 @@
+"""ctypes binding of libvscan.so: argument marshalling only.
+
+Each function mirrors one entry point of include/vscan.h, takes CUDA torch tensors (used purely
+as device memory) and enqueues the library's kernels on torch's current stream.  There is no
+fallback of any kind: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import _build
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+F32, BF16 = 0, 1
+SCORE_ROW, SCORE_QK = 0, 1
+SPAN_ONLY, SPAN_FULL = 0, 1
+MERGE_AUTO, MERGE_SIMT, MERGE_TENSOR = 0, 1, 2
+
+_vp, _i32, _f32 = C.c_void_p, C.c_int32, C.c_float
+
+
+class ScoreDesc(C.Structure):
+    _fields_ = [("mode", _i32), ("dtype", _i32), ("attn", _vp), ("instances", _i32), ("heads", _i32),
+                ("row_len", _i32), ("cls_offset", _i32), ("n_tokens", _i32), ("q", _vp), ("k", _vp),
+                ("batch", _i32), ("q_heads", _i32), ("kv_heads", _i32), ("seq_len", _i32),
+                ("head_dim", _i32), ("span_begin", _i32), ("span_len", _i32), ("softmax_span", _i32),
+                ("scale", _f32), ("scores", _vp)]
+
+
+class SelectDesc(C.Structure):
+    _fields_ = [("scores_global", _vp), ("scores_local", _vp), ("instances", _i32), ("frames", _i32),
+                ("grid_h", _i32), ("grid_w", _i32), ("win_h", _i32), ("win_w", _i32),
+                ("k_per_window", _i32), ("k_global", _i32), ("kept_idx", _vp), ("kept_mask", _vp)]
+
+
+class MergeDesc(C.Structure):
+    _fields_ = [("dtype", _i32), ("path", _i32), ("x", _vp), ("metric", _vp), ("kept_idx", _vp),
+                ("instances", _i32), ("row_len", _i32), ("cls_offset", _i32), ("n_tokens", _i32),
+                ("dim", _i32), ("metric_dim", _i32), ("n_kept", _i32), ("merged", _vp), ("assign", _vp),
+                ("counts", _vp)]
+
+
+class PruneDesc(C.Structure):
+    _fields_ = [("dtype", _i32), ("q_last", _vp), ("k", _vp), ("v", _vp), ("hidden", _vp),
+                ("pos_ids", _vp), ("batch", _i32), ("q_heads", _i32), ("kv_heads", _i32),
+                ("head_dim", _i32), ("hidden_dim", _i32), ("pos_planes", _i32), ("n_sys", _i32),
+                ("n_vis", _i32), ("n_txt", _i32), ("k_keep", _i32), ("softmax_span", _i32),
+                ("scale", _f32), ("kept_vis", _vp), ("hidden_out", _vp), ("k_out", _vp), ("v_out", _vp),
+                ("pos_out", _vp), ("scores", _vp)]
+
+
+class VScanError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status}, cuda error {lib().vscan_last_cuda_error()})")
+
+
+_LIB = None
+
+
+def lib() -> C.CDLL:
+    """Load libvscan.so (building it first if the sources are newer).  Raises if unavailable."""
+    global _LIB
+    if _LIB is None:
+        path = _build.LIB_PATH
+        if not os.path.exists(path) or os.environ.get("VSCAN_REBUILD") == "1":
+            path = _build.build()
+        L = C.CDLL(path)
+        for name, desc in (("score", ScoreDesc), ("select", SelectDesc), ("merge", MergeDesc),
+                           ("llm_prune", PruneDesc)):
+            ws = getattr(L, f"vscan_{name}_workspace_bytes")
+            ws.restype, ws.argtypes = C.c_size_t, [C.POINTER(desc)]
+        for fn, desc in (("vscan_score", ScoreDesc), ("vscan_select_global_local", SelectDesc),
+                         ("vscan_merge", MergeDesc), ("vscan_llm_prune", PruneDesc)):
+            f = getattr(L, fn)
+            f.restype, f.argtypes = _i32, [C.POINTER(desc), _vp, C.c_size_t, _vp]
+        L.vscan_version.restype = _i32
+        L.vscan_status_string.restype, L.vscan_status_string.argtypes = C.c_char_p, [_i32]
+        L.vscan_check.restype, L.vscan_check.argtypes = _i32, [_vp, _vp]
+        L.vscan_last_cuda_error.restype = _i32
+        L.vscan_kernel_launches.restype = C.c_uint64
+        _LIB = L
+    return _LIB
+
+
+def status_string(status: int) -> str:
+    return lib().vscan_status_string(status).decode()
+
+
+def kernel_launches() -> int:
+    return int(lib().vscan_kernel_launches())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Workspace:
+    """A reusable device scratch buffer (256-byte aligned by the torch allocator)."""
+
+    def __init__(self, nbytes: int = 0, device="cuda"):
+        self.device = device
+        self.buf = None
+        self.reserve(nbytes)
+
+    def reserve(self, nbytes: int):
+        if self.buf is None or self.buf.numel() < nbytes:
+            self.buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.device)
+        return self
+
+    @property
+    def ptr(self):
+        return self.buf.data_ptr()
+
+    @property
+    def nbytes(self):
+        return self.buf.numel()
+
+
+def _call(fn_name, desc, ws_fn_name, workspace):
+    L = lib()
+    need = getattr(L, ws_fn_name)(C.byref(desc))
+    if workspace is None:
+        workspace = Workspace(need)
+    elif workspace.nbytes < need:
+        raise VScanError(ERR_WORKSPACE, f"{fn_name}: workspace of {workspace.nbytes} B < {need} B")
+    st = getattr(L, fn_name)(C.byref(desc), workspace.ptr, workspace.nbytes, _stream())
+    if st != OK:
+        raise VScanError(st, fn_name)
+    return workspace
+
+
+# ------------------------------------------------------------------------------------------ API
+def score_row_desc(attn, cls_offset, n_tokens, scores) -> ScoreDesc:
+    B, H, L = attn.shape
+    return ScoreDesc(mode=SCORE_ROW, dtype=_dtype_code(attn), attn=_ptr(attn), instances=B, heads=H,
+                     row_len=L, cls_offset=cls_offset, n_tokens=n_tokens, scores=_ptr(scores))
+
+
+def vscan_score_row(attn: torch.Tensor, cls_offset: int, n_tokens: int | None = None,
+                    out: torch.Tensor | None = None) -> torch.Tensor:
+    """Eq. 2: head mean of attention rows.  attn [B', H, L] -> scores [B', N] float32."""
+    n = attn.shape[2] - cls_offset if n_tokens is None else n_tokens
+    if out is None:
+        out = torch.empty((attn.shape[0], n), dtype=torch.float32, device=attn.device)
+    d = score_row_desc(attn, cls_offset, n, out)
+    st = lib().vscan_score(C.byref(d), None, 0, _stream())
+    if st != OK:
+        raise VScanError(st, "vscan_score")
+    return out
+
+
+def score_qk_desc(q, k, span_begin, span_len, scale, softmax_span, scores) -> ScoreDesc:
+    B, Hq, d = q.shape
+    _, Hkv, S, _ = k.shape
+    return ScoreDesc(mode=SCORE_QK, dtype=_dtype_code(k), q=_ptr(q), k=_ptr(k), batch=B, q_heads=Hq,
+                     kv_heads=Hkv, seq_len=S, head_dim=d, span_begin=span_begin, span_len=span_len,
+                     softmax_span=softmax_span, scale=scale, scores=_ptr(scores))
+
+
+def vscan_score_qk(q, k, span_begin, span_len, scale, softmax_span=SPAN_ONLY, out=None, workspace=None):
+    """Eq. 5: head mean of softmax(scale * q . K) on a span.  -> scores [B, span_len] float32."""
+    if out is None:
+        out = torch.empty((q.shape[0], span_len), dtype=torch.float32, device=q.device)
+    d = score_qk_desc(q, k, span_begin, span_len, scale, softmax_span, out)
+    _call("vscan_score", d, "vscan_score_workspace_bytes", workspace)
+    return out
+
+
+def vscan_select_global_local(scores_global, scores_local, frames, grid_h, grid_w, win_h, win_w,
+                              k_per_window, k_global, out=None, want_mask=False):
+    """Sec. 4.1 selection.  -> kept_idx [B', K1] int32 ascending (and the optional uint8 mask)."""
+    B = scores_global.shape[0]
+    windows = frames * (grid_h // max(win_h, 1)) * (grid_w // max(win_w, 1))
+    k1 = windows * k_per_window + k_global
+    if out is None:
+        out = torch.empty((B, max(k1, 0)), dtype=torch.int32, device=scores_global.device)
+    mask = torch.empty((B, frames * grid_h * grid_w), dtype=torch.uint8, device=out.device) if want_mask else None
+    d = SelectDesc(scores_global=_ptr(scores_global), scores_local=_ptr(scores_local), instances=B,
+                   frames=frames, grid_h=grid_h, grid_w=grid_w, win_h=win_h, win_w=win_w,
+                   k_per_window=k_per_window, k_global=k_global, kept_idx=_ptr(out), kept_mask=_ptr(mask))
+    st = lib().vscan_select_global_local(C.byref(d), None, 0, _stream())
+    if st != OK:
+        raise VScanError(st, "vscan_select_global_local")
+    return (out, mask) if want_mask else out
+
+
+def vscan_merge(x, cls_offset, kept_idx, n_tokens=None, metric=None, path=MERGE_AUTO, out=None,
+                want_assign=False, want_counts=False, workspace=None):
+    """Eq. 4.  x [B', L, D], kept_idx [B', K1] -> merged [B', K1, D] (+ assign, counts)."""
+    B, L, D = x.shape
+    n = L - cls_offset if n_tokens is None else n_tokens
+    K1 = kept_idx.shape[1]
+    if out is None:
+        out = torch.empty((B, K1, D), dtype=x.dtype, device=x.device)
+    assign = torch.empty((B, n), dtype=torch.int32, device=x.device) if want_assign else None
+    counts = torch.empty((B, K1), dtype=torch.int32, device=x.device) if want_counts else None
+    d = MergeDesc(dtype=_dtype_code(x), path=path, x=_ptr(x), metric=_ptr(metric), kept_idx=_ptr(kept_idx),
+                  instances=B, row_len=L, cls_offset=cls_offset, n_tokens=n, dim=D,
+                  metric_dim=0 if metric is None else metric.shape[2], n_kept=K1, merged=_ptr(out),
+                  assign=_ptr(assign), counts=_ptr(counts))
+    _call("vscan_merge", d, "vscan_merge_workspace_bytes", workspace)
+    res = [out]
+    if want_assign:
+        res.append(assign)
+    if want_counts:
+        res.append(counts)
+    return res[0] if len(res) == 1 else tuple(res)
+
+
+def vscan_llm_prune(q_last, k, v, hidden, pos_ids, n_sys, n_vis, n_txt, k_keep, scale,
+                    softmax_span=SPAN_ONLY, want_scores=False, out=None, workspace=None):
+    """Sec. 4.2.  Returns a dict with kept_vis, hidden, k, v, pos (and scores)."""
+    B, Hq, d_ = q_last.shape
+    Hkv = k.shape[1]
+    S = n_sys + n_vis + n_txt
+    So = S - n_vis + k_keep
+    dev = k.device
+    o = out or {}
+    o.setdefault("kept_vis", torch.empty((B, k_keep), dtype=torch.int32, device=dev))
+    o.setdefault("k", torch.empty((B, Hkv, So, d_), dtype=k.dtype, device=dev))
+    if v is not None:
+        o.setdefault("v", torch.empty((B, Hkv, So, d_), dtype=v.dtype, device=dev))
+    if hidden is not None:
+        o.setdefault("hidden", torch.empty((B, So, hidden.shape[2]), dtype=hidden.dtype, device=dev))
+    if pos_ids is not None:
+        o.setdefault("pos", torch.empty((pos_ids.shape[0], B, So), dtype=torch.int32, device=dev))
+    if want_scores:
+        o.setdefault("scores", torch.empty((B, n_vis), dtype=torch.float32, device=dev))
+    desc = PruneDesc(dtype=_dtype_code(k), q_last=_ptr(q_last), k=_ptr(k), v=_ptr(v), hidden=_ptr(hidden),
+                     pos_ids=_ptr(pos_ids), batch=B, q_heads=Hq, kv_heads=Hkv, head_dim=d_,
+                     hidden_dim=0 if hidden is None else hidden.shape[2],
+                     pos_planes=0 if pos_ids is None else pos_ids.shape[0], n_sys=n_sys, n_vis=n_vis,
+                     n_txt=n_txt, k_keep=k_keep, softmax_span=softmax_span, scale=scale,
+                     kept_vis=_ptr(o["kept_vis"]), hidden_out=_ptr(o.get("hidden")), k_out=_ptr(o["k"]),
+                     v_out=_ptr(o.get("v")), pos_out=_ptr(o.get("pos")), scores=_ptr(o.get("scores")))
+    _call("vscan_llm_prune", desc, "vscan_llm_prune_workspace_bytes", workspace)
+    return o
+
+
+def vscan_check(workspace: Workspace) -> int:
+    return int(lib().vscan_check(workspace.ptr, _stream()))

@@ -1,0 +1,341 @@
+// vscan_merge: cosine arg-max assignment of the unselected tokens and mean merge (Eq. 4).
+//   kept_inv_norm_kernel   1 / max(|m_s|, eps) of every kept token
+//   assign (SIMT or tensor) a(u) = argmax_s (m_u . m_s) * inv_norm[s]   (|m_u| is constant along a
+//                           row of the similarity matrix and cannot change the arg-max)
+//   group_mean_kernel      members of every slot in ascending token order, fp32 sum, one rounding
+#include "merge.cuh"
+
+namespace vscan {
+
+// ------------------------------------------------------------------ norms of the kept tokens
+// One warp per kept token.  grid = (ceil(n_kept / 8), instances), 256 threads.
+template <typename T>
+__global__ void __launch_bounds__(256) kept_inv_norm_kernel(MergeParams p) {
+  constexpr int E = Vec16<T>::kElems;
+  const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *p.status = 0u;
+  if (s >= p.n_kept) return;
+  int t = p.kept[static_cast<size_t>(b) * p.n_kept + s];
+  t = min(max(t, 0), p.n_tokens - 1);
+  const uint4* row = reinterpret_cast<const uint4*>(
+      static_cast<const T*>(p.metric) + (static_cast<size_t>(b) * p.row_len + p.cls_offset + t) * p.metric_dim);
+  const int vecs = p.metric_dim / E;
+  float ss = 0.f;
+  for (int v = lane; v < vecs; v += 32) {
+    float f[E];
+    Vec16<T>::unpack(ld_nc_16(row + v), f);
+#pragma unroll
+    for (int e = 0; e < E; ++e) ss = fmaf(f[e], f[e], ss);
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) p.inv_norm[static_cast<size_t>(b) * p.n_kept + s] = 1.f / fmaxf(sqrtf(ss), 1e-12f);
+}
+
+// ------------------------------------------------------------------ assignment on CUDA cores
+// CTA tile: 64 tokens x 64 kept, 32-wide slices of the feature dim, 4x4 outputs per thread.
+constexpr int kTileT = 64, kTileS = 64, kTileK = 32, kPad = 4;
+
+template <typename T>
+__global__ void __launch_bounds__(256) assign_simt_kernel(MergeParams p) {
+  constexpr int E = Vec16<T>::kElems;
+  constexpr int kVecPerRow = kTileK / E;
+  __shared__ __align__(16) float As[kTileK][kTileT + kPad];
+  __shared__ __align__(16) float Bs[kTileK][kTileS + kPad];
+  __shared__ int kept_row[kTileS];
+  __shared__ float kept_scale[kTileS];
+  __shared__ int best_slot[kTileT];
+
+  const int b = blockIdx.y, t0 = blockIdx.x * kTileT;
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const T* mb = static_cast<const T*>(p.metric) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.metric_dim;
+  const int32_t* kept = p.kept + static_cast<size_t>(b) * p.n_kept;
+  const float* inv_norm = p.inv_norm + static_cast<size_t>(b) * p.n_kept;
+
+  float run_val[4];
+  int run_idx[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { run_val[i] = -INFINITY; run_idx[i] = 0; }
+
+  for (int s0 = 0; s0 < p.n_kept; s0 += kTileS) {
+    __syncthreads();
+    if (threadIdx.x < kTileS) {
+      int s = s0 + threadIdx.x;
+      int t = s < p.n_kept ? min(max(kept[s], 0), p.n_tokens - 1) : -1;
+      kept_row[threadIdx.x] = t;
+      kept_scale[threadIdx.x] = s < p.n_kept ? inv_norm[s] : 0.f;
+    }
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = 0; k0 < p.metric_dim; k0 += kTileK) {
+      __syncthreads();
+      for (int idx = threadIdx.x; idx < kTileT * kVecPerRow; idx += 256) {
+        const int row = idx / kVecPerRow, vec = idx % kVecPerRow, kk = k0 + vec * E;
+        float fa[E], fb[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) { fa[e] = 0.f; fb[e] = 0.f; }
+        const int t = t0 + row;
+        if (t < p.n_tokens && kk < p.metric_dim)
+          Vec16<T>::unpack(ld_nc_16(mb + static_cast<size_t>(t) * p.metric_dim + kk), fa);
+        const int tk = kept_row[row];
+        if (tk >= 0 && kk < p.metric_dim)
+          Vec16<T>::unpack(ld_nc_16(mb + static_cast<size_t>(tk) * p.metric_dim + kk), fb);
+#pragma unroll
+        for (int e = 0; e < E; ++e) { As[vec * E + e][row] = fa[e]; Bs[vec * E + e][row] = fb[e]; }
+      }
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < kTileK; ++k) {
+        const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+        const float4 c = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+        const float av[4] = {a.x, a.y, a.z, a.w}, cv[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], cv[j], acc[i][j]);
+      }
+    }
+    // arg-max of this kept tile, lowest slot on ties
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float bv = -INFINITY;
+      int bi = 0x7fffffff;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int s = s0 + tx * 4 + j;
+        if (s < p.n_kept) {
+          const float v = acc[i][j] * kept_scale[tx * 4 + j];
+          if (v > bv) { bv = v; bi = s; }
+        }
+      }
+#pragma unroll
+      for (int o = 1; o < 16; o <<= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
+      }
+      if (bv > run_val[i]) { run_val[i] = bv; run_idx[i] = bi; }
+    }
+  }
+  if (tx == 0) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) best_slot[ty * 4 + i] = run_idx[i] == 0x7fffffff ? 0 : run_idx[i];
+  }
+  __syncthreads();
+  // a kept token belongs to its own slot
+  for (int s = threadIdx.x; s < p.n_kept; s += 256) {
+    const int t = min(max(kept[s], 0), p.n_tokens - 1);
+    if (t >= t0 && t < t0 + kTileT) best_slot[t - t0] = s;
+  }
+  __syncthreads();
+  if (threadIdx.x < kTileT && t0 + threadIdx.x < p.n_tokens)
+    p.assign[static_cast<size_t>(b) * p.n_tokens + t0 + threadIdx.x] = best_slot[threadIdx.x];
+}
+
+vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t stream) {
+  dim3 grid((p.n_tokens + kTileT - 1) / kTileT, p.instances);
+  if (dtype == VSCAN_F32) assign_simt_kernel<float><<<grid, 256, 0, stream>>>(p);
+  else assign_simt_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(p);
+  VSCAN_AFTER_LAUNCH();
+  return VSCAN_OK;
+}
+
+// ------------------------------------------------------------------ group means
+// One CTA per (group of 8 slots, instance); warp w owns slot s0 + w.  The CTA first lists, in
+// ascending token order, the tokens assigned to its 8 slots; each warp then walks that list and
+// adds its members' rows in that order (fp32), two rows in flight.
+// dynamic shared memory: list[n_tokens] of (local slot << 24 | token)
+constexpr int kSlotsPerCta = 8;
+
+template <typename T, int VPL>
+__global__ void __launch_bounds__(256) group_mean_kernel(MergeParams p) {
+  constexpr int E = Vec16<T>::kElems;
+  extern __shared__ __align__(16) uint32_t list[];
+  __shared__ int warp_sums[33];
+  const int b = blockIdx.y, s0 = blockIdx.x * kSlotsPerCta;
+  const int32_t* assign = p.assign + static_cast<size_t>(b) * p.n_tokens;
+
+  const int per = (p.n_tokens + blockDim.x - 1) / blockDim.x;
+  const int lo = min(p.n_tokens, static_cast<int>(threadIdx.x) * per), hi = min(p.n_tokens, lo + per);
+  int mine = 0;
+  for (int i = lo; i < hi; ++i) {
+    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
+    mine += rel < static_cast<unsigned>(kSlotsPerCta);
+  }
+  int n_list;
+  int pos = block_exclusive_scan(mine, warp_sums, n_list);
+  for (int i = lo; i < hi; ++i) {
+    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
+    if (rel < static_cast<unsigned>(kSlotsPerCta)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
+  }
+  __syncthreads();
+
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, s = s0 + w;
+  if (s >= p.n_kept) return;
+  const int vecs = p.dim / E;
+  const T* xb = static_cast<const T*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
+  T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
+
+  for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
+    float acc[VPL][E];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+    int count = 0;
+    for (int c = 0; c < n_list; c += 32) {
+      const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
+      unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(w));
+      count += __popc(mask);
+      while (mask) {
+        const int l0 = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const int l1 = mask ? __ffs(mask) - 1 : -1;
+        if (mask) mask &= mask - 1;
+        const int ta = static_cast<int>(__shfl_sync(0xffffffffu, entry, l0) & 0xFFFFFFu);
+        const int tb = l1 >= 0 ? static_cast<int>(__shfl_sync(0xffffffffu, entry, l1) & 0xFFFFFFu) : -1;
+        const uint4* ra = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(ta) * p.dim);
+        const uint4* rb = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tb < 0 ? ta : tb) * p.dim);
+        uint4 va[VPL], vb[VPL];
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+          const int v = v0 + lane + 32 * i;
+          if (v < vecs) { va[i] = ld_nc_16(ra + v); if (tb >= 0) vb[i] = ld_nc_16(rb + v); }
+        }
+#pragma unroll
+        for (int i = 0; i < VPL; ++i) {
+          const int v = v0 + lane + 32 * i;
+          if (v < vecs) {
+            float f[E];
+            Vec16<T>::unpack(va[i], f);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+            if (tb >= 0) {
+              Vec16<T>::unpack(vb[i], f);
+#pragma unroll
+              for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+            }
+          }
+        }
+      }
+    }
+    const float inv = 1.f / static_cast<float>(max(count, 1));
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      const int v = v0 + lane + 32 * i;
+      if (v < vecs) {
+        float f[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
+        st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
+      }
+    }
+    if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
+  }
+}
+
+template <typename T>
+static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream) {
+  constexpr int E = Vec16<T>::kElems;
+  const size_t smem = static_cast<size_t>(p.n_tokens) * 4 + 16;
+  if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
+  dim3 grid((p.n_kept + kSlotsPerCta - 1) / kSlotsPerCta, p.instances);
+  if (p.dim / E <= 128) {
+    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4>, smem));
+    group_mean_kernel<T, 4><<<grid, 256, smem, stream>>>(p);
+  } else {
+    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8>, smem));
+    group_mean_kernel<T, 8><<<grid, 256, smem, stream>>>(p);
+  }
+  VSCAN_AFTER_LAUNCH();
+  return VSCAN_OK;
+}
+
+}  // namespace vscan
+
+using namespace vscan;
+
+static vscan_status validate_merge(const vscan_merge_desc* d) {
+  if (!d || !d->x || !d->kept_idx || !d->merged) return VSCAN_ERR_INVALID_ARG;
+  if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
+  if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR)
+    return VSCAN_ERR_INVALID_ARG;
+  if (d->instances < 0 || d->n_tokens <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + d->n_tokens ||
+      d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
+    return VSCAN_ERR_INVALID_ARG;
+  if (d->metric && (d->metric_dim <= 0 || d->metric_dim % 8)) return VSCAN_ERR_INVALID_ARG;
+  if (d->n_tokens >= (1 << 24)) return VSCAN_ERR_UNSUPPORTED;
+  if (d->instances > 65535) return VSCAN_ERR_UNSUPPORTED;
+  const void* ptrs[] = {d->x, d->metric, d->kept_idx, d->merged, d->assign, d->counts};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return VSCAN_ERR_INVALID_ARG;
+  const size_t e = dtype_bytes(d->dtype), B = d->instances;
+  struct Rng { const void* p; size_t n; };
+  const Rng ins[] = {{d->x, B * d->row_len * d->dim * e},
+                     {d->metric, d->metric ? B * d->row_len * d->metric_dim * e : 0},
+                     {d->kept_idx, B * d->n_kept * 4}};
+  const Rng outs[] = {{d->merged, B * d->n_kept * d->dim * e}, {d->assign, B * d->n_tokens * 4},
+                      {d->counts, B * d->n_kept * 4}};
+  for (const Rng& o : outs) {
+    for (const Rng& i : ins)
+      if (overlaps(o.p, o.n, i.p, i.n)) return VSCAN_ERR_INVALID_ARG;
+    for (const Rng& o2 : outs)
+      if (o.p != o2.p && overlaps(o.p, o.n, o2.p, o2.n)) return VSCAN_ERR_INVALID_ARG;
+  }
+  return VSCAN_OK;
+}
+
+extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
+  if (!d || d->instances <= 0 || d->n_kept <= 0 || d->n_tokens <= 0) return kStatusBytes;
+  size_t bytes = kStatusBytes;
+  bytes += round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256);    // inv_norm
+  bytes += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);  // assign
+  return bytes;
+}
+
+extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, size_t workspace_bytes,
+                                    void* stream_) {
+  vscan_status st = validate_merge(d);
+  if (st != VSCAN_OK) return st;
+  if (d->instances == 0) return VSCAN_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const size_t need = vscan_merge_workspace_bytes(d);
+  if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
+
+  MergeParams p;
+  p.x = d->x;
+  p.metric = d->metric ? d->metric : d->x;
+  p.metric_dim = d->metric ? d->metric_dim : d->dim;
+  p.kept = d->kept_idx;
+  char* ws = static_cast<char*>(workspace);
+  p.status = reinterpret_cast<uint32_t*>(ws);
+  p.inv_norm = reinterpret_cast<float*>(ws + kStatusBytes);
+  int32_t* ws_assign = reinterpret_cast<int32_t*>(
+      ws + kStatusBytes + round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256));
+  p.assign = d->assign ? d->assign : ws_assign;
+  p.merged = d->merged; p.counts = d->counts;
+  p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
+  p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
+
+  bool tensor = false;
+  if (d->path == VSCAN_MERGE_TENSOR) {
+    if (!assign_tensor_supported(d->dtype, p)) return VSCAN_ERR_UNSUPPORTED;
+    tensor = true;
+  } else if (d->path == VSCAN_MERGE_AUTO) {
+    tensor = assign_tensor_supported(d->dtype, p);
+  }
+
+  dim3 ngrid((d->n_kept + 7) / 8, d->instances);
+  if (d->dtype == VSCAN_F32) kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p);
+  else kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p);
+  VSCAN_AFTER_LAUNCH();
+
+  st = tensor ? launch_assign_tensor(p, stream) : launch_assign_simt(d->dtype, p, stream);
+  if (st != VSCAN_OK) return st;
+
+  return d->dtype == VSCAN_F32 ? launch_group_mean<float>(p, stream)
+                               : launch_group_mean<__nv_bfloat16>(p, stream);
+}

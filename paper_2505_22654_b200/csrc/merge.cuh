@@ -1,0 +1,27 @@
+// Internal declarations of the merge step (Sec. 4.1 "Token Merging", Eq. 4).
+#pragma once
+
+#include "common.cuh"
+
+namespace vscan {
+
+struct MergeParams {
+  const void* x;        // [instances][row_len][dim]
+  const void* metric;   // [instances][row_len][metric_dim] (== x when no separate metric)
+  const int32_t* kept;  // [instances][n_kept]
+  float* inv_norm;      // [instances][n_kept]   1 / max(|m_kept|, 1e-12)       (workspace)
+  int32_t* assign;      // [instances][n_tokens]                                  (workspace or output)
+  void* merged;         // [instances][n_kept][dim]
+  int32_t* counts;      // optional
+  uint32_t* status;     // device status word
+  int instances, row_len, cls_offset, n_tokens, dim, metric_dim, n_kept;
+};
+
+// Similarity contraction + arg-max on CUDA cores (fp32 FMA).  Works for both dtypes.
+vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t stream);
+// Same result on the tensor cores (bf16 only).  Returns VSCAN_ERR_UNSUPPORTED for shapes it
+// cannot take.
+vscan_status launch_assign_tensor(const MergeParams& p, cudaStream_t stream);
+bool assign_tensor_supported(int dtype, const MergeParams& p);
+
+}  // namespace vscan

@@ -1,0 +1,129 @@
+// vscan_score: head-mean of attention rows (ROW mode, Eq. 2) and of softmax(q.K) (QK mode, Eq. 5).
+#include "score.cuh"
+
+namespace vscan {
+
+// ROW mode.  grid = (ceil(n_tokens / blockDim), instances); one thread per token, heads ascending.
+template <typename T>
+__global__ void __launch_bounds__(256) row_mean_kernel(const T* __restrict__ attn, float* __restrict__ scores,
+                                                       int heads, int row_len, int cls_offset, int n_tokens) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n_tokens) return;
+  const T* base = attn + static_cast<size_t>(blockIdx.y) * heads * row_len + cls_offset + j;
+  float acc = 0.f;
+  int h = 0;
+  for (; h + 4 <= heads; h += 4) {
+    float a0 = to_float(base[static_cast<size_t>(h) * row_len]);
+    float a1 = to_float(base[static_cast<size_t>(h + 1) * row_len]);
+    float a2 = to_float(base[static_cast<size_t>(h + 2) * row_len]);
+    float a3 = to_float(base[static_cast<size_t>(h + 3) * row_len]);
+    acc += a0; acc += a1; acc += a2; acc += a3;
+  }
+  for (; h < heads; ++h) acc += to_float(base[static_cast<size_t>(h) * row_len]);
+  scores[static_cast<size_t>(blockIdx.y) * n_tokens + j] = acc / static_cast<float>(heads);
+}
+
+__global__ void head_mean_kernel(const float* __restrict__ probs, float* __restrict__ scores, int q_heads,
+                                 int span_len) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= span_len) return;
+  const float* base = probs + static_cast<size_t>(blockIdx.y) * q_heads * span_len + j;
+  float acc = 0.f;
+  for (int h = 0; h < q_heads; ++h) acc += base[static_cast<size_t>(h) * span_len];
+  scores[static_cast<size_t>(blockIdx.y) * span_len + j] = acc / static_cast<float>(q_heads);
+}
+
+vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStream_t stream) {
+  const size_t smem = qk_smem_bytes(p.head_dim, p.soft_n);
+  if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
+  dim3 grid(p.q_heads, batch);
+  if (dtype == VSCAN_F32) {
+    VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<float>, smem));
+    qk_softmax_kernel<float><<<grid, 256, smem, stream>>>(p);
+  } else {
+    VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<__nv_bfloat16>, smem));
+    qk_softmax_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(p);
+  }
+  VSCAN_AFTER_LAUNCH();
+  return VSCAN_OK;
+}
+
+}  // namespace vscan
+
+using namespace vscan;
+
+static vscan_status validate_score(const vscan_score_desc* d) {
+  if (!d || !d->scores) return VSCAN_ERR_INVALID_ARG;
+  if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
+  if (!aligned16(d->scores)) return VSCAN_ERR_INVALID_ARG;
+  const size_t e = dtype_bytes(d->dtype);
+  if (d->mode == VSCAN_SCORE_ROW) {
+    if (!d->attn || !aligned16(d->attn)) return VSCAN_ERR_INVALID_ARG;
+    if (d->instances < 0 || d->heads <= 0 || d->n_tokens < 0 || d->cls_offset < 0 ||
+        d->row_len < d->cls_offset + d->n_tokens)
+      return VSCAN_ERR_INVALID_ARG;
+    if (overlaps(d->scores, static_cast<size_t>(d->instances) * d->n_tokens * 4, d->attn,
+                 static_cast<size_t>(d->instances) * d->heads * d->row_len * e))
+      return VSCAN_ERR_INVALID_ARG;
+    return VSCAN_OK;
+  }
+  if (d->mode == VSCAN_SCORE_QK) {
+    if (!d->q || !d->k || !aligned16(d->q) || !aligned16(d->k)) return VSCAN_ERR_INVALID_ARG;
+    if (d->batch < 0 || d->q_heads <= 0 || d->kv_heads <= 0 || d->q_heads % d->kv_heads ||
+        d->seq_len <= 0 || d->head_dim <= 0 || d->span_begin < 0 || d->span_len < 0 ||
+        d->span_begin + d->span_len > d->seq_len)
+      return VSCAN_ERR_INVALID_ARG;
+    if (d->softmax_span != VSCAN_SPAN_ONLY && d->softmax_span != VSCAN_SPAN_FULL)
+      return VSCAN_ERR_INVALID_ARG;
+    if (d->head_dim % 8 || d->head_dim > 256) return VSCAN_ERR_INVALID_ARG;
+    if (overlaps(d->scores, static_cast<size_t>(d->batch) * d->span_len * 4, d->k,
+                 static_cast<size_t>(d->batch) * d->kv_heads * d->seq_len * d->head_dim * e) ||
+        overlaps(d->scores, static_cast<size_t>(d->batch) * d->span_len * 4, d->q,
+                 static_cast<size_t>(d->batch) * d->q_heads * d->head_dim * e))
+      return VSCAN_ERR_INVALID_ARG;
+    return VSCAN_OK;
+  }
+  return VSCAN_ERR_INVALID_ARG;
+}
+
+extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
+  if (!d || d->mode != VSCAN_SCORE_QK || d->batch <= 0 || d->q_heads <= 0 || d->span_len <= 0) return 0;
+  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * d->q_heads * d->span_len * sizeof(float), 256);
+}
+
+extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, size_t workspace_bytes,
+                                    void* stream_) {
+  vscan_status st = validate_score(d);
+  if (st != VSCAN_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (d->mode == VSCAN_SCORE_ROW) {
+    if (d->instances == 0 || d->n_tokens == 0) return VSCAN_OK;
+    dim3 grid((d->n_tokens + 255) / 256, d->instances);
+    if (d->dtype == VSCAN_F32)
+      row_mean_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(d->attn), d->scores, d->heads,
+                                                       d->row_len, d->cls_offset, d->n_tokens);
+    else
+      row_mean_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(d->attn),
+                                                               d->scores, d->heads, d->row_len, d->cls_offset,
+                                                               d->n_tokens);
+    VSCAN_AFTER_LAUNCH();
+    return VSCAN_OK;
+  }
+  if (d->batch == 0 || d->span_len == 0) return VSCAN_OK;
+  const size_t need = vscan_score_workspace_bytes(d);
+  if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
+  QkParams p;
+  p.q = d->q; p.k = d->k;
+  p.status = static_cast<uint32_t*>(workspace);
+  p.probs = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+  p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = d->seq_len; p.head_dim = d->head_dim;
+  p.span_begin = d->span_begin; p.span_len = d->span_len; p.scale = d->scale;
+  if (d->softmax_span == VSCAN_SPAN_ONLY) { p.soft_lo = d->span_begin; p.soft_n = d->span_len; }
+  else { p.soft_lo = 0; p.soft_n = d->seq_len; }
+  st = launch_qk_softmax(d->dtype, p, d->batch, stream);
+  if (st != VSCAN_OK) return st;
+  dim3 grid((d->span_len + 255) / 256, d->batch);
+  head_mean_kernel<<<grid, 256, 0, stream>>>(p.probs, d->scores, d->q_heads, d->span_len);
+  VSCAN_AFTER_LAUNCH();
+  return VSCAN_OK;
+}

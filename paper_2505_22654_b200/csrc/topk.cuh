@@ -1,0 +1,116 @@
+// Exact top-k selection on order-preserving uint32 keys held in shared memory.
+//
+// "k largest, equal keys to the lowest index" is found in two steps: a radix select yields the
+// threshold T (the k-th largest key among the candidates) and `need`, the number of candidates
+// equal to T that still belong to the set; every key above T is taken, and of the keys equal to
+// T the first `need` in index order.  No sort, no float atomics, exactly k survivors.
+#pragma once
+
+#include "common.cuh"
+
+namespace vscan {
+
+struct SelectScratch {
+  int hist[256];
+  int warp_sums[33];
+  uint32_t threshold;
+  int need;
+};
+
+// Block-wide radix select, 4 passes of 8 bits.  Candidates are the i in [0, n) with
+// excluded == nullptr || !excluded[i].  Requires 1 <= k <= #candidates.  All threads of the
+// block must call; on return every thread reads the same (threshold, need).
+__device__ __forceinline__ void block_radix_select(const uint32_t* keys, const uint8_t* excluded, int n,
+                                                   int k, SelectScratch& sc, uint32_t& threshold,
+                                                   int& need) {
+  uint32_t prefix = 0, mask = 0;
+  int k_rem = k;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) sc.hist[i] = 0;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      if (excluded && excluded[i]) continue;
+      uint32_t key = keys[i];
+      if ((key & mask) == prefix) atomicAdd(&sc.hist[(key >> shift) & 255u], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      // lane l owns bins [8l, 8l+8); walk from the top bin down
+      const int lane = threadIdx.x;
+      int local[8], sum = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { local[j] = sc.hist[lane * 8 + j]; sum += local[j]; }
+      // above = candidates in bins owned by higher lanes
+      int incl = sum;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        int t = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += t;
+      }
+      int above = incl - sum;
+      // the k_rem-th largest lies in this lane's bins iff above < k_rem <= above + sum
+      if (above < k_rem && k_rem <= above + sum) {
+        int acc = above;
+#pragma unroll
+        for (int j = 7; j >= 0; --j) {
+          if (acc < k_rem && k_rem <= acc + local[j]) {
+            sc.threshold = prefix | (static_cast<uint32_t>(lane * 8 + j) << shift);
+            sc.need = k_rem - acc;
+          }
+          acc += local[j];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = sc.threshold;
+    k_rem = sc.need;
+    mask |= 0xFFu << shift;
+    __syncthreads();
+  }
+  threshold = prefix;
+  need = k_rem;
+}
+
+// Warp-wide bitwise select over m candidates enumerated by `token_of(p)`, p in [0, m), ascending
+// in p.  Marks the k winners in `selected` (shared memory, one byte per token).  0 <= k <= m.
+template <typename TokenOf>
+__device__ __forceinline__ void warp_select_mark(const uint32_t* keys, int m, int k, TokenOf token_of,
+                                                 uint8_t* selected) {
+  if (k <= 0) return;
+  const int lane = threadIdx.x & 31;
+  uint32_t prefix = 0;
+  int k_rem = k;
+  for (int bit = 31; bit >= 0; --bit) {
+    const uint32_t hi_mask = ~((2u << bit) - 1u);  // bits above `bit`; 0 when bit == 31
+    int cnt = 0;
+    for (int p0 = 0; p0 < m; p0 += 32) {
+      int p = p0 + lane;
+      bool hit = false;
+      if (p < m) {
+        uint32_t key = keys[token_of(p)];
+        hit = ((key & hi_mask) == prefix) && ((key >> bit) & 1u);
+      }
+      cnt += __popc(__ballot_sync(0xffffffffu, hit));
+    }
+    if (cnt >= k_rem) prefix |= (1u << bit); else k_rem -= cnt;
+  }
+  // prefix is the k-th largest key; k_rem of the keys equal to it belong to the set
+  int taken_eq = 0;
+  for (int p0 = 0; p0 < m; p0 += 32) {
+    int p = p0 + lane;
+    bool gt = false, eq = false;
+    int t = 0;
+    if (p < m) {
+      t = token_of(p);
+      uint32_t key = keys[t];
+      gt = key > prefix;
+      eq = key == prefix;
+    }
+    unsigned eq_mask = __ballot_sync(0xffffffffu, eq);
+    int rank = taken_eq + __popc(eq_mask & ((1u << lane) - 1u));
+    if (gt || (eq && rank < k_rem)) selected[t] = 1;
+    taken_eq += __popc(eq_mask);
+  }
+}
+
+}  // namespace vscan

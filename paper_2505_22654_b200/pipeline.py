@@ -1,0 +1,95 @@
+"""Chained Stage 1 + Stage 2 reduction with preallocated buffers (argument marshalling only).
+
+`VScanReducer` owns the output tensors and workspaces for one fixed shape so that a pass makes no
+allocation and can be captured in a CUDA graph.  `run_host` is the end-to-end form: inputs arrive
+in pinned host memory, results are returned in pinned host memory.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as vb
+
+
+class VScanReducer:
+    def __init__(self, *, dtype, instances, frames, grid_h, grid_w, cls, D, H, win_h, win_w, k_w, k_g,
+                 B, n_sys, n_vis, n_txt, Dh, Hq, Hkv, d, k2, pos_planes=1, scale=None,
+                 softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, device="cuda"):
+        self.dtype = torch.float32 if dtype in ("f32", torch.float32) else torch.bfloat16
+        self.instances, self.frames, self.grid_h, self.grid_w, self.cls = instances, frames, grid_h, grid_w, cls
+        self.D, self.H, self.win_h, self.win_w, self.k_w, self.k_g = D, H, win_h, win_w, k_w, k_g
+        self.N = frames * grid_h * grid_w
+        self.L = self.N + cls
+        self.W = frames * (grid_h // win_h) * (grid_w // win_w)
+        self.K1 = k_g + self.W * k_w
+        self.B, self.n_sys, self.n_vis, self.n_txt = B, n_sys, n_vis, n_txt
+        self.Dh, self.Hq, self.Hkv, self.d, self.k2, self.P = Dh, Hq, Hkv, d, k2, pos_planes
+        self.S = n_sys + n_vis + n_txt
+        self.S_out = self.S - n_vis + k2
+        self.scale = float(scale if scale is not None else d ** -0.5)
+        self.softmax_span, self.merge_path = softmax_span, merge_path
+        dev, dt = device, self.dtype
+        self.scores_g = torch.empty((instances, self.N), dtype=torch.float32, device=dev)
+        self.scores_l = torch.empty((instances, self.N), dtype=torch.float32, device=dev)
+        self.kept_idx = torch.empty((instances, self.K1), dtype=torch.int32, device=dev)
+        self.merged = torch.empty((instances, self.K1, D), dtype=dt, device=dev)
+        self.out2 = {
+            "kept_vis": torch.empty((B, k2), dtype=torch.int32, device=dev),
+            "hidden": torch.empty((B, self.S_out, Dh), dtype=dt, device=dev),
+            "k": torch.empty((B, Hkv, self.S_out, d), dtype=dt, device=dev),
+            "v": torch.empty((B, Hkv, self.S_out, d), dtype=dt, device=dev),
+            "pos": torch.empty((pos_planes, B, self.S_out), dtype=torch.int32, device=dev),
+        }
+        self.ws_merge = vb.Workspace(64 << 10, dev)
+        self.ws_prune = vb.Workspace(64 << 10, dev)
+        self._sized = False
+
+    @classmethod
+    def from_config(cls_, cfg, **kw):
+        return cls_(dtype=cfg.dtype, instances=cfg.instances, frames=cfg.frames, grid_h=cfg.grid_h,
+                    grid_w=cfg.grid_w, cls=cfg.cls, D=cfg.D, H=cfg.H, win_h=cfg.win_h, win_w=cfg.win_w,
+                    k_w=cfg.k_w, k_g=cfg.k_g, B=cfg.B, n_sys=cfg.n_sys, n_vis=cfg.n_vis, n_txt=cfg.n_txt,
+                    Dh=cfg.Dh, Hq=cfg.Hq, Hkv=cfg.Hkv, d=cfg.d, k2=cfg.k2, pos_planes=cfg.pos_planes, **kw)
+
+    # ---- device-resident pass: the four library calls on the current stream
+    def stage1(self, attn_g, attn_l, x):
+        vb.vscan_score_row(attn_g, self.cls, self.N, out=self.scores_g)
+        vb.vscan_score_row(attn_l, self.cls, self.N, out=self.scores_l)
+        vb.vscan_select_global_local(self.scores_g, self.scores_l, self.frames, self.grid_h, self.grid_w,
+                                     self.win_h, self.win_w, self.k_w, self.k_g, out=self.kept_idx)
+        if not self._sized:
+            self._reserve(x)
+        vb.vscan_merge(x, self.cls, self.kept_idx, n_tokens=self.N, path=self.merge_path, out=self.merged,
+                       workspace=self.ws_merge)
+        return self.merged
+
+    def stage2(self, q_last, k, v, hidden, pos_ids):
+        return vb.vscan_llm_prune(q_last, k, v, hidden, pos_ids, self.n_sys, self.n_vis, self.n_txt, self.k2,
+                                  self.scale, self.softmax_span, out=self.out2, workspace=self.ws_prune)
+
+    def run(self, attn_g, attn_l, x, q_last, k, v, hidden, pos_ids):
+        self.stage1(attn_g, attn_l, x)
+        return self.stage2(q_last, k, v, hidden, pos_ids)
+
+    def _reserve(self, x):
+        import ctypes as C
+        L = vb.lib()
+        md = vb.MergeDesc(dtype=vb._dtype_code(x), instances=self.instances, n_kept=self.K1, n_tokens=self.N,
+                          dim=self.D, row_len=self.L, cls_offset=self.cls)
+        self.ws_merge.reserve(L.vscan_merge_workspace_bytes(C.byref(md)))
+        pd = vb.PruneDesc(batch=self.B, q_heads=self.Hq, n_vis=self.n_vis)
+        self.ws_prune.reserve(L.vscan_llm_prune_workspace_bytes(C.byref(pd)))
+        self._sized = True
+
+    # ---- end to end: pinned host buffers in, pinned host buffers out
+    def run_host(self, host_in: dict, host_out: dict, dev_in: dict):
+        """host_in / dev_in: same keys (attn_g, attn_l, x, q_last, k, v, hidden, pos_ids); host_out:
+        merged, kept_vis, hidden, k, v, pos.  Copies in, runs the pass, copies out, all on the
+        current stream; the caller synchronises."""
+        for name, t in host_in.items():
+            dev_in[name].copy_(t, non_blocking=True)
+        self.run(**dev_in)
+        host_out["merged"].copy_(self.merged, non_blocking=True)
+        for name in ("kept_vis", "hidden", "k", "v", "pos"):
+            host_out[name].copy_(self.out2[name], non_blocking=True)
+        return host_out

@@ -1,0 +1,224 @@
+"""Per-call parity of the CUDA library against the CPU oracle on small and edge-case shapes
+(several tiles plus ragged tails).  Everything goes through the C ABI via the ctypes binding."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2505_22654_b200 as vs
+from oracle import plant
+from oracle import vscan_oracle as vo
+from synth import CONFIGS, round_to_dtype
+
+from helpers import TOL_SCORE, check_merged, dev, stage1_case, stage2_case
+
+pytestmark = pytest.mark.gpu
+RNG = np.random.default_rng(7)
+
+
+def small_cfg(dtype, **kw):
+    base = CONFIGS[2].with_(name="small", config_id=50, B=2, C=3, grid_h=12, grid_w=18, D=72, H=5, k_w=2,
+                            k_g=9, n_clusters=6, n_sys=3, n_txt=5, Dh=72, Hq=6, Hkv=3, d=40, k2=17, dtype=dtype)
+    return base.with_(**kw)
+
+
+# ------------------------------------------------------------------ vscan_score, ROW mode
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("B,H,L,c", [(1, 1, 9, 1), (3, 16, 577, 1), (2, 7, 300, 0), (2, 3, 1031, 1)])
+def test_score_row(dtype, B, H, L, c):
+    attn = round_to_dtype(RNG.random((B, H, L)).astype(np.float32) / L, dtype)
+    got = vs.vscan_score_row(dev(attn, dtype), c).cpu().numpy()
+    ref = np.stack([vo.score_row(attn[b], c) for b in range(B)])
+    assert got.shape == ref.shape
+    assert np.abs(got - ref).max() <= TOL_SCORE
+
+
+def test_score_row_partial_row_and_empty_batch():
+    attn = RNG.random((2, 4, 50)).astype(np.float32)
+    got = vs.vscan_score_row(dev(attn, "f32"), 2, n_tokens=40).cpu().numpy()
+    ref = np.stack([vo.score_row(attn[b][:, :42], 2) for b in range(2)])
+    assert np.abs(got - ref).max() <= 1e-6
+    empty = torch.empty((0, 4, 50), device="cuda")
+    assert vs.vscan_score_row(empty, 1).shape == (0, 49)
+
+
+# ------------------------------------------------------------------ vscan_select_global_local
+SELECT_SHAPES = [  # F, Gh, Gw, wh, ww, k_w, k_g
+    (1, 24, 24, 6, 6, 2, 32), (1, 24, 24, 6, 6, 6, 96), (1, 24, 24, 6, 6, 0, 64), (1, 24, 24, 6, 6, 3, 0),
+    (1, 24, 24, 24, 24, 10, 5), (2, 4, 6, 2, 3, 1, 3), (1, 1, 1, 1, 1, 1, 0), (1, 5, 7, 1, 1, 0, 35),
+    (3, 10, 10, 5, 2, 4, 100), (16, 32, 32, 8, 8, 4, 1024), (1, 24, 24, 6, 6, 36, 0), (4, 16, 16, 16, 16, 37, 11),
+]
+
+
+@pytest.mark.parametrize("shape", SELECT_SHAPES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_select_bit_exact(shape, ties):
+    F, Gh, Gw, wh, ww, k_w, k_g = shape
+    N, B = F * Gh * Gw, 3
+    if ties:   # few distinct values, signed zeros and negatives: the tie rule decides nearly everything
+        sg = RNG.integers(-2, 3, (B, N)).astype(np.float32) * 0.25
+        sl = RNG.integers(0, 3, (B, N)).astype(np.float32) * 0.5
+        sg[:, ::7] = -0.0
+    else:
+        sg = RNG.random((B, N)).astype(np.float32)
+        sl = RNG.standard_normal((B, N)).astype(np.float32)
+    got, mask = vs.vscan_select_global_local(dev(sg), dev(sl), F, Gh, Gw, wh, ww, k_w, k_g, want_mask=True)
+    got, mask = got.cpu().numpy(), mask.cpu().numpy()
+    for b in range(B):
+        ref = vo.select_global_local(sg[b], sl[b], F, Gh, Gw, wh, ww, k_w, k_g)[0]
+        np.testing.assert_array_equal(got[b], ref)
+        m = np.zeros(N, dtype=np.uint8); m[ref] = 1
+        np.testing.assert_array_equal(mask[b], m)
+
+
+def test_select_uniform_scores_take_first_indices_and_aliasing():
+    s = dev(np.full((2, 576), 0.125, dtype=np.float32))
+    got = vs.vscan_select_global_local(s, s, 1, 24, 24, 6, 6, 2, 32).cpu().numpy()
+    ref = vo.select_global_local(np.full(576, 0.125), np.full(576, 0.125), 1, 24, 24, 6, 6, 2, 32)[0]
+    np.testing.assert_array_equal(got[0], ref); np.testing.assert_array_equal(got[1], ref)
+    # window w starts at row 6*(w//4), column 6*(w%4): its first two tokens are kept
+    assert {0, 1, 6, 7, 144, 145}.issubset(set(got[0].tolist()))
+
+
+# ------------------------------------------------------------------ vscan_merge
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("path", ["simt", "auto"])
+def test_merge_small_planted(dtype, path):
+    cfg = small_cfg(dtype)
+    case = stage1_case(cfg)
+    x, kept = dev(case["x"], dtype), dev(case["kept"].astype(np.int32))
+    merged, assign, counts = vs.vscan_merge(x, cfg.cls, kept, want_assign=True, want_counts=True,
+                                            path=vs.MERGE_SIMT if path == "simt" else vs.MERGE_AUTO)
+    np.testing.assert_array_equal(assign.cpu().numpy(), case["assign"])
+    np.testing.assert_array_equal(counts.cpu().numpy(), case["counts"])
+    check_merged(merged, case["merged"], dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_merge_edge_shapes(dtype):
+    D, L, c = 264, 131, 1
+    N = L - c
+    x = round_to_dtype(RNG.standard_normal((2, L, D)).astype(np.float32), dtype)
+    xd = dev(x, dtype)
+    # keep-all: identity, bit for bit
+    kept_all = np.tile(np.arange(N, dtype=np.int32), (2, 1))
+    merged, counts = vs.vscan_merge(xd, c, dev(kept_all), want_counts=True)
+    assert torch.equal(merged, xd[:, c:]) and int(counts.min()) == 1 == int(counts.max())
+    # a single kept token receives the mean of everything
+    one = np.array([[5], [77]], dtype=np.int32)
+    merged, assign, counts = vs.vscan_merge(xd, c, dev(one), want_assign=True, want_counts=True)
+    assert int(assign.abs().max()) == 0 and counts.flatten().tolist() == [N, N]
+    ref = x[:, c:].astype(np.float64).mean(axis=1, keepdims=True)
+    check_merged(merged, ref, dtype)
+    # ragged kept count (not a multiple of the tile) with margins planted
+    cfg = small_cfg(dtype, grid_h=10, grid_w=13, win_h=10, win_w=13, k_w=0, k_g=67, D=264, C=1, B=2)
+    x2 = round_to_dtype(RNG.standard_normal((2, cfg.L, D)).astype(np.float32), dtype)
+    kept = np.stack([np.sort(RNG.choice(cfg.N, 67, replace=False)) for _ in range(2)])
+    plant.plant_merge(cfg, x2, kept)
+    merged, assign, counts = vs.vscan_merge(dev(x2, dtype), cfg.cls, dev(kept.astype(np.int32)),
+                                            want_assign=True, want_counts=True)
+    for b in range(2):
+        m, a, cn = vo.merge(x2[b], cfg.cls, kept[b])
+        np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
+        np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
+        check_merged(merged[b], m, dtype)
+
+
+def test_merge_exact_ties_and_duplicates():
+    # identical tokens: every cosine ties at 1 -> lowest slot; kept duplicates keep their own slot
+    x = np.tile(RNG.standard_normal((1, 1, 16)).astype(np.float32), (1, 40, 1))
+    kept = np.array([[3, 10, 25]], dtype=np.int32)
+    merged, assign, counts = vs.vscan_merge(dev(x, "f32"), 0, dev(kept), want_assign=True, want_counts=True)
+    ref_m, ref_a, ref_c = vo.merge(x[0], 0, kept[0])
+    np.testing.assert_array_equal(assign[0].cpu().numpy(), ref_a)
+    assert counts[0].tolist() == ref_c.tolist() == [38, 1, 1]
+    # a zero vector has cosine 0 with everything -> slot 0
+    x2 = RNG.standard_normal((1, 12, 8)).astype(np.float32); x2[0, 4] = 0
+    kept2 = np.array([[1, 7]], dtype=np.int32)
+    _, a2 = vs.vscan_merge(dev(x2, "f32"), 0, dev(kept2), want_assign=True)
+    np.testing.assert_array_equal(a2[0].cpu().numpy(), vo.merge(x2[0], 0, kept2[0])[1])
+    assert int(a2[0, 4]) == 0
+
+
+def test_merge_separate_metric():
+    x = RNG.standard_normal((2, 50, 24)).astype(np.float32)
+    metric = RNG.standard_normal((2, 50, 16)).astype(np.float32)
+    kept = np.stack([np.sort(RNG.choice(50, 6, replace=False)) for _ in range(2)]).astype(np.int32)
+    merged, assign = vs.vscan_merge(dev(x, "f32"), 0, dev(kept), metric=dev(metric, "f32"), want_assign=True)
+    for b in range(2):
+        m, a, _ = vo.merge(x[b], 0, kept[b], metric=metric[b])
+        np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
+        check_merged(merged[b], m, "f32")
+
+
+# ------------------------------------------------------------------ vscan_score, QK mode
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("span", [vo.SPAN_ONLY, vo.SPAN_FULL])
+@pytest.mark.parametrize("B,Hq,Hkv,S,d,b0,n", [(2, 6, 3, 70, 40, 3, 51), (1, 32, 32, 139, 128, 35, 64),
+                                               (2, 28, 4, 300, 128, 0, 257), (1, 4, 1, 9, 8, 8, 1)])
+def test_score_qk(dtype, span, B, Hq, Hkv, S, d, b0, n):
+    q = round_to_dtype(RNG.standard_normal((B, Hq, d)).astype(np.float32), dtype)
+    k = round_to_dtype(RNG.standard_normal((B, Hkv, S, d)).astype(np.float32), dtype)
+    scale = 1.0 / np.sqrt(d)
+    got = vs.vscan_score_qk(dev(q, dtype), dev(k, dtype), b0, n, scale, span).cpu().numpy()
+    ref = np.stack([vo.score_qk(q[b], k[b], b0, n, float(np.float32(scale)), span) for b in range(B)])
+    assert np.abs(got - ref).max() <= TOL_SCORE
+    if span == vo.SPAN_ONLY:
+        np.testing.assert_allclose(got.sum(-1), 1.0, atol=1e-5)
+
+
+# ------------------------------------------------------------------ vscan_llm_prune
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("span", [vo.SPAN_ONLY, vo.SPAN_FULL])
+def test_llm_prune_small_planted(dtype, span):
+    cfg = small_cfg(dtype, pos_planes=3)
+    case = stage2_case(cfg, softmax_span=span)
+    case["pos_ids"][1] *= 3; case["pos_ids"][2] += 100            # planes differ
+    out = vs.vscan_llm_prune(dev(case["q_last"], dtype), dev(case["k"], dtype), dev(case["v"], dtype),
+                             dev(case["hidden"], dtype), dev(case["pos_ids"]), cfg.n_sys, cfg.n_vis, cfg.n_txt,
+                             cfg.k2, case["scale"], span, want_scores=True)
+    o = case["oracle"]
+    assert np.abs(out["scores"].cpu().numpy() - o["scores"]).max() <= TOL_SCORE
+    np.testing.assert_array_equal(out["kept_vis"].cpu().numpy(), o["kept_vis"])
+    for name in ("hidden", "k", "v"):
+        np.testing.assert_array_equal(out[name].float().cpu().numpy(), o[name])      # bit-exact copies
+    for b in range(cfg.B):
+        rows = vo.compaction_rows(cfg.n_sys, cfg.n_vis, cfg.n_txt, o["kept_vis"][b])
+        np.testing.assert_array_equal(out["pos"][:, b].cpu().numpy(), case["pos_ids"][:, b][:, rows])
+
+
+@pytest.mark.parametrize("k_keep,n_sys,n_txt", [(0, 3, 4), (20, 3, 4), (7, 0, 0), (20, 0, 5), (1, 2, 0)])
+def test_llm_prune_edges(k_keep, n_sys, n_txt):
+    n_vis, Hq, Hkv, d, Dh, B = 20, 4, 2, 16, 24, 2
+    S = n_sys + n_vis + n_txt
+    q = RNG.standard_normal((B, Hq, d)).astype(np.float32)
+    k = RNG.standard_normal((B, Hkv, S, d)).astype(np.float32)
+    v = RNG.standard_normal((B, Hkv, S, d)).astype(np.float32)
+    h = RNG.standard_normal((B, S, Dh)).astype(np.float32)
+    pos = np.tile(np.arange(S, dtype=np.int32) * 2, (1, B, 1))
+    out = vs.vscan_llm_prune(dev(q), dev(k), dev(v), dev(h), dev(pos), n_sys, n_vis, n_txt, k_keep, 0.25)
+    for b in range(B):
+        o = vo.llm_prune(q[b], k[b], v[b], h[b], pos[:, b], n_sys, n_vis, n_txt, k_keep, 0.25)
+        np.testing.assert_array_equal(out["kept_vis"][b].cpu().numpy(), o["kept_vis"])
+        np.testing.assert_array_equal(out["hidden"][b].cpu().numpy(), o["hidden"])
+        np.testing.assert_array_equal(out["k"][b].cpu().numpy(), o["k"])
+        np.testing.assert_array_equal(out["v"][b].cpu().numpy(), o["v"])
+        np.testing.assert_array_equal(out["pos"][:, b].cpu().numpy(), o["pos"])
+        assert np.all(np.diff(out["pos"][0, b].cpu().numpy()) > 0)
+    # K only (no V, hidden or position ids)
+    out2 = vs.vscan_llm_prune(dev(q), dev(k), None, None, None, n_sys, n_vis, n_txt, k_keep, 0.25)
+    assert torch.equal(out2["k"], out["k"]) and "v" not in out2
+
+
+def test_workspace_too_small_and_status_word():
+    cfg = small_cfg("bf16")
+    case = stage2_case(cfg, planted=False)
+    args = (dev(case["q_last"], "bf16"), dev(case["k"], "bf16"), None, None, None, cfg.n_sys, cfg.n_vis,
+            cfg.n_txt, cfg.k2, case["scale"])
+    with pytest.raises(vs.VScanError) as e:
+        vs.vscan_llm_prune(*args, workspace=vs.Workspace(256))
+    assert e.value.status == 3
+    ws = vs.Workspace(1 << 20)
+    ws.buf.fill_(0xFF)
+    vs.vscan_llm_prune(*args, workspace=ws)
+    assert vs.vscan_check(ws) == 0
+    assert vs.kernel_launches() > 0
