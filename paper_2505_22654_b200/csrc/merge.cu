@@ -298,6 +298,7 @@ extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
 
 extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, size_t workspace_bytes,
                                     void* stream_) {
+  if (d && d->instances == 0) return VSCAN_OK;  // empty batch
   vscan_status st = validate_merge(d);
   if (st != VSCAN_OK) return st;
   if (d->instances == 0) return VSCAN_OK;

@@ -133,7 +133,8 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
 using namespace vscan;
 
 static vscan_status validate_prune(const vscan_prune_desc* d) {
-  if (!d || !d->q_last || !d->k || !d->kept_vis || !d->k_out) return VSCAN_ERR_INVALID_ARG;
+  if (!d || !d->q_last || !d->k || !d->k_out) return VSCAN_ERR_INVALID_ARG;
+  if (!d->kept_vis && d->k_keep > 0) return VSCAN_ERR_INVALID_ARG;  // an empty survivor list may be NULL
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
   if ((d->v == nullptr) != (d->v_out == nullptr) || (d->hidden == nullptr) != (d->hidden_out == nullptr) ||
       (d->pos_ids == nullptr) != (d->pos_out == nullptr))
@@ -177,6 +178,7 @@ extern "C" size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* d) {
 
 extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspace, size_t workspace_bytes,
                                         void* stream_) {
+  if (d && d->batch == 0) return VSCAN_OK;  // empty batch
   vscan_status st = validate_prune(d);
   if (st != VSCAN_OK) return st;
   if (d->batch == 0) return VSCAN_OK;

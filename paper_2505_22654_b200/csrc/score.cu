@@ -93,6 +93,8 @@ extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
 
 extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, size_t workspace_bytes,
                                     void* stream_) {
+  if (d && ((d->mode == VSCAN_SCORE_ROW && d->instances == 0) || (d->mode == VSCAN_SCORE_QK && d->batch == 0)))
+    return VSCAN_OK;  // empty batch: nothing to read or write
   vscan_status st = validate_score(d);
   if (st != VSCAN_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);

@@ -94,6 +94,7 @@ extern "C" size_t vscan_select_workspace_bytes(const vscan_select_desc*) { retur
 
 extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
                                                   size_t /*workspace_bytes*/, void* stream) {
+  if (d && d->instances == 0) return VSCAN_OK;  // empty batch
   if (!d || !d->scores_global || !d->scores_local || !d->kept_idx) return VSCAN_ERR_INVALID_ARG;
   if (d->instances < 0 || d->frames <= 0 || d->grid_h <= 0 || d->grid_w <= 0 || d->win_h <= 0 ||
       d->win_w <= 0)
