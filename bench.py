@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the VScan reduction path (Stage 1 + Stage 2) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl vscan|reference]
+
+One step = one pass of the whole path (score x2 -> select -> merge -> prune) over one batch of the
+LLaVA-NeXT workload (32 images x 5 crops x 576 patches = 2880 visual tokens per image, bf16).
+Prints one JSON line.  `value` is images/s with inputs resident in HBM (CUDA-graph replays, CUDA
+events, max over ranks); `e2e` is the same pass with pinned-host inputs copied in and results copied
+out inside the timed region; `roofline` is the dominant kernel's algorithmic bytes over its CUDA-event
+duration against the measured HBM copy bandwidth; `cpu_baseline` is the numpy oracle on the host.
+With N > 1 every rank runs an independent replica of the batch (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from synth import CONFIGS, stage1_inputs, stage2_inputs, sweep_config  # noqa: E402
+
+METRIC = "VScan reduction images/s (Stage1+Stage2) at 2880 visual tokens"
+UNIT = "images/s"
+FALLBACK_HBM_GBS = 6650.0
+MERGE_KERNELS = ("kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", "merge_fused")
+
+
+# ------------------------------------------------------------------ algorithmic work per step
+def algorithmic_bytes(cfg) -> dict:
+    """Bytes each call has to move per step (whole batch): inputs read once, outputs written once."""
+    e, I, B = cfg.elem_bytes, cfg.instances, cfg.B
+    row = {
+        "row_mean": I * (cfg.H * cfg.L * e + cfg.N * 4),                       # one launch (two per step)
+        "select": I * (2 * cfg.N * 4 + cfg.K1 * 4),
+        "merge": I * (cfg.N * cfg.D * e + cfg.K1 * 4 + cfg.K1 * cfg.D * e),     # X once + merged out
+        "qk_softmax": B * (cfg.Hkv * cfg.n_vis * cfg.d * e + cfg.Hq * cfg.d * e),
+        "prune_topk": B * cfg.k2 * 4,
+        "compact": B * 2 * cfg.S_out * (cfg.Dh * e + 2 * cfg.Hkv * cfg.d * e + cfg.pos_planes * 4),
+    }
+    row["step"] = 2 * row["row_mean"] + row["select"] + row["merge"] + row["qk_softmax"] + \
+        row["prune_topk"] + row["compact"]
+    return row
+
+
+def merge_flops(cfg) -> float:
+    return 2.0 * cfg.instances * (cfg.N - cfg.K1) * cfg.K1 * cfg.D
+
+
+def measured_peaks() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(path))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks during the timed region
+class ClockSampler(threading.Thread):
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, device_index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reason_bits, self.max_mhz = period_s, [], 0, None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _reasons(self):
+        for fn in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            f = getattr(self.nv, fn, None)
+            if f is not None:
+                try:
+                    return int(f(self.h))
+                except Exception:
+                    pass
+        return 0
+
+    def sample_once(self):
+        try:
+            self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            self.reason_bits |= self._reasons()
+        except Exception:
+            pass
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._stop_evt.is_set():
+            self.sample_once()
+            time.sleep(self.period)
+
+    def finish(self) -> dict:
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ oracle timing (CPU baseline)
+def oracle_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_image(cfg, s1, s2, img: int):
+    """The whole path for one image on the CPU oracle: its C crops through Stage 1, its sequence
+    through Stage 2."""
+    from oracle import vscan_oracle as vo
+    for c in range(cfg.C):
+        i = img * cfg.C + c
+        sg = vo.score_row(s1["attn_g"][i], cfg.cls)
+        sl = vo.score_row(s1["attn_l"][i], cfg.cls)
+        kept = vo.select_global_local(sg, sl, cfg.frames, cfg.grid_h, cfg.grid_w, cfg.win_h, cfg.win_w,
+                                      cfg.k_w, cfg.k_g)[0]
+        vo.merge(s1["x"][i], cfg.cls, kept)
+    vo.llm_prune(s2["q_last"][img], s2["k"][img], s2["v"][img], s2["hidden"][img], s2["pos_ids"][:, img],
+                 cfg.n_sys, cfg.n_vis, cfg.n_txt, cfg.k2, s2["scale"])
+
+
+def time_oracle(cfg, budget_s: float = 12.0, max_images: int = 16):
+    n = min(cfg.B, max_images)
+    s1 = stage1_inputs(cfg, 0, n * cfg.C)
+    s2 = stage2_inputs(cfg, 0, n)
+    oracle_image(cfg, s1, s2, 0)            # warm numpy / BLAS
+    done, t0 = 0, time.perf_counter()
+    while True:
+        oracle_image(cfg, s1, s2, done % n)
+        done += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s or done >= 4 * n:
+            break
+    return {"value": done / el, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "sample": f"{done} images of the {cfg.name} workload ({cfg.C} crops + 1 sequence each), "
+                      f"{el:.1f} s of numpy fp64"}
+
+
+def run_reference(args, cfg):
+    """The oracle as the reference arm: one image of the workload per step."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    n = 4
+    s1 = stage1_inputs(cfg, 0, n * cfg.C)
+    s2 = stage2_inputs(cfg, 0, n)
+    for w in range(max(args.warmup, 1)):
+        oracle_image(cfg, s1, s2, w % n)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        oracle_image(cfg, s1, s2, i % n)
+    el = time.perf_counter() - t0
+    value = args.steps / el
+    sample = f"1 image ({cfg.C} crops + 1 sequence) of the workload per step, numpy fp64 oracle on the host"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "images_per_step": 1},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ multi-rank plumbing
+def dist_setup(n_gpus: int):
+    """-> (rank, world, local_rank, dist or None).  One process per GPU under torchrun."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world <= 1:
+        return 0, 1, 0, None
+    import torch.distributed as dist
+    dist.init_process_group(os.environ.get("VSCAN_BENCH_BACKEND", "nccl"))
+    return dist.get_rank(), world, int(os.environ.get("LOCAL_RANK", "0")), dist
+
+
+def max_over_ranks(value_ms: float, dist, device) -> float:
+    if dist is None:
+        return value_ms
+    import torch
+    t = torch.tensor([value_ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------ the GPU arm
+def build_sets(cfg, n_sets: int, device):
+    """Generate one batch on the host (at most 32 distinct images, tiled beyond that); the other sets
+    are the same batch with the images rotated, so that consecutive steps touch different memory."""
+    import torch
+    dt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    gen_b = min(cfg.B, 32)
+    s1, s2 = stage1_inputs(cfg, 0, gen_b * cfg.C), stage2_inputs(cfg, 0, gen_b)
+
+    def tile(a, total, axis=0):
+        reps = -(-total // a.shape[axis])
+        return np.concatenate([a] * reps, axis=axis).take(range(total), axis=axis) if reps > 1 else a
+
+    host = {"attn_g": tile(s1["attn_g"], cfg.instances), "attn_l": tile(s1["attn_l"], cfg.instances),
+            "x": tile(s1["x"], cfg.instances), "q_last": tile(s2["q_last"], cfg.B), "k": tile(s2["k"], cfg.B),
+            "v": tile(s2["v"], cfg.B), "hidden": tile(s2["hidden"], cfg.B)}
+    sets = []
+    for r in range(n_sets):
+        d = {}
+        for name, a in host.items():
+            shift = r * (cfg.C if name in ("attn_g", "attn_l", "x") else 1)
+            d[name] = torch.from_numpy(np.roll(a, shift, axis=0)).to(device=device, dtype=dt).contiguous()
+        d["pos_ids"] = torch.from_numpy(tile(s2["pos_ids"], cfg.B, axis=1)).to(device).contiguous()
+        sets.append(d)
+    return sets
+
+
+def run_vscan(args, cfg):
+    import torch
+
+    import paper_2505_22654_b200 as vs
+    from paper_2505_22654_b200 import binding as vb
+
+    rank, world, local_rank, dist = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the VScan path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    vb.lib()
+
+    n_sets = args.sets
+    warmup = max(args.warmup, 3)
+    sets = build_sets(cfg, n_sets, device)
+    reducers = [vs.VScanReducer.from_config(cfg, device=device, merge_path=args.merge_path) for _ in range(n_sets)]
+    stream = torch.cuda.Stream(device)
+    launches_per_step = 0
+    with torch.cuda.stream(stream):
+        for w in range(warmup):
+            before = vs.kernel_launches()
+            reducers[w % n_sets].run(**sets[w % n_sets])
+            launches_per_step = vs.kernel_launches() - before
+        stream.synchronize()
+        graphs = []
+        if not args.no_graph:
+            for r in range(n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    reducers[r].run(**sets[r])
+                graphs.append(g)
+            for i in range(warmup):
+                graphs[i % n_sets].replay()
+            stream.synchronize()
+
+        def step(i):
+            if graphs:
+                graphs[i % n_sets].replay()
+            else:
+                reducers[i % n_sets].run(**sets[i % n_sets])
+
+        # ---- timed region: exactly K steps between barriers and synchronisations
+        sampler = ClockSampler(local_rank)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        sampler.start()
+        ev0.record(stream)
+        for i in range(args.steps):
+            step(i)
+        ev1.record(stream)
+        if sampler.ok:
+            sampler.sample_once()       # at least one sample while the queue is still draining
+        ev1.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.finish()
+        if dist is not None:
+            dist.barrier()
+        ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, device)
+
+        # ---- per-kernel durations: the same steps launched directly, each kernel between two events
+        prof_steps = max(1, min(args.steps, 30))
+        cap = prof_steps * launches_per_step + 8
+        vb.profile_begin(cap)
+        for i in range(prof_steps):
+            reducers[i % n_sets].run(**sets[i % n_sets])
+        records = vb.profile_end(cap)
+        per_kernel = {}
+        for name, ms in records:
+            per_kernel.setdefault(name, []).append(ms)
+
+        # ---- end to end: pinned host buffers in and out, copies inside the timed region
+        red, dev_in = reducers[0], sets[0]
+        host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in dev_in.items()}
+        outs = {"merged": red.merged, **{k: red.out2[k] for k in ("kept_vis", "hidden", "k", "v", "pos")}}
+        host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
+        e_steps = max(1, min(args.steps, 5))
+        red.run_host(host_in, host_out, dev_in)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(e_steps):
+            red.run_host(host_in, host_out, dev_in)
+        e1.record(stream)
+        e1.synchronize()
+        e_ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
+        e2e = {"value": world * cfg.B * e_steps / (e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in.values())),
+               "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out.values())),
+               "steps": e_steps, "ms_per_step": e_ms / e_steps}
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        alg = algorithmic_bytes(cfg)
+        ms_step = ms_total / args.steps
+        kernels = {}
+        total_k = sum(sum(v) for v in per_kernel.values())
+        for name, v in per_kernel.items():
+            kernels[name] = {"launches_per_step": len(v) / prof_steps, "avg_us": 1e3 * float(np.mean(v)),
+                             "share": sum(v) / total_k}
+        merge_names = [n for n in kernels if n in MERGE_KERNELS]
+        dominant = max(kernels, key=lambda n: kernels[n]["share"])
+        # the merge call is several kernels that share one pass over the features: its algorithmic
+        # bytes are charged to whichever of them is being reported
+        dom_bytes = alg["merge"] if dominant in merge_names else alg[dominant]
+        achieved = dom_bytes / (kernels[dominant]["avg_us"] * 1e-6) / 1e9
+        traffic = None
+        try:
+            traffic = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json"))).get(dominant)
+        except Exception:
+            pass
+        cpu = time_oracle(cfg) if (world == 1 and not args.no_cpu_baseline) else None
+        step_gbs = alg["step"] / (ms_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": world * cfg.B * args.steps / (ms_total * 1e-3), "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": cfg.dtype,
+            "data": "synthetic",
+            "config": {"workload": cfg.name, "images_per_step": cfg.B, "crops_per_image": cfg.C,
+                       "visual_tokens_per_image": cfg.C * cfg.N, "kept_per_crop": cfg.K1, "stage2_keep": cfg.k2,
+                       "launch": "cuda graph replay" if graphs else "stream launches",
+                       "l2": f"inputs+outputs {alg['step'] / 1e6:.0f} MB per step > 126 MB L2; "
+                             f"{n_sets} rotating buffer sets",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "step_hbm": {"algorithmic_bytes": alg["step"], "achieved_gbs": step_gbs, "frac": step_gbs / peak,
+                         "peak_gbs": peak, "peak_kind": peak_kind},
+            "roofline": {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                         "algorithmic_bytes_per_launch": dom_bytes},
+            "kernels": kernels,
+            "merge": {"flops_per_step": merge_flops(cfg),
+                      "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names)},
+            "gpu_launches": launches_per_step * args.steps,
+            "clocks": clocks,
+            "e2e": e2e,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="vscan", choices=["vscan", "reference"])
+    ap.add_argument("--workload", default="2", help="0-3, or sweep:<batch>:<retention>")
+    ap.add_argument("--sets", type=int, default=3, help="rotating buffer sets")
+    ap.add_argument("--merge-path", type=int, default=0, help="0 auto, 1 CUDA cores, 2 tensor cores")
+    ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.workload.startswith("sweep:"):
+        _, b, r = args.workload.split(":")
+        cfg = sweep_config(int(b), r)
+    else:
+        cfg = CONFIGS[int(args.workload)]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_vscan(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -211,6 +211,15 @@ vscan_status vscan_llm_prune(const vscan_prune_desc* desc, void* workspace, size
  * vscan_kernel_launches: number of kernels this library has launched in this process so far.
  * ------------------------------------------------------------------------------------------- */
 int32_t vscan_version(void);
+/* Per-kernel timing, a measurement aid with no counterpart in the paper.  Between
+ * vscan_profile_begin(capacity) and vscan_profile_end every kernel the library launches is bracketed
+ * by two CUDA events on its stream (up to `capacity` launches; later ones are not recorded).
+ * vscan_profile_end waits for the recorded launches, writes for each, in launch order, a
+ * NUL-terminated kernel name into names[i*32 .. i*32+31] and its duration in milliseconds into
+ * millis[i] (both host arrays of `capacity` entries), releases the events and returns the count
+ * (-1 if profiling was not on).  Do not use while a stream is being captured into a graph. */
+vscan_status vscan_profile_begin(int32_t capacity);
+int32_t vscan_profile_end(char* names, float* millis, int32_t capacity);
 const char* vscan_status_string(vscan_status status);
 vscan_status vscan_check(const void* workspace, void* stream);
 int32_t vscan_last_cuda_error(void);

@@ -82,6 +82,9 @@ def lib() -> C.CDLL:
         L.vscan_check.restype, L.vscan_check.argtypes = _i32, [_vp, _vp]
         L.vscan_last_cuda_error.restype = _i32
         L.vscan_kernel_launches.restype = C.c_uint64
+        L.vscan_profile_begin.restype, L.vscan_profile_begin.argtypes = _i32, [_i32]
+        L.vscan_profile_end.restype = _i32
+        L.vscan_profile_end.argtypes = [C.c_char_p, C.POINTER(C.c_float), _i32]
         _LIB = L
     return _LIB
 
@@ -255,6 +258,23 @@ def vscan_llm_prune(q_last, k, v, hidden, pos_ids, n_sys, n_vis, n_txt, k_keep, 
                      v_out=_ptr(o.get("v")), pos_out=_ptr(o.get("pos")), scores=_ptr(o.get("scores")))
     _call("vscan_llm_prune", desc, "vscan_llm_prune_workspace_bytes", workspace)
     return o
+
+
+def profile_begin(capacity: int = 4096):
+    st = lib().vscan_profile_begin(capacity)
+    if st != OK:
+        raise VScanError(st, "vscan_profile_begin")
+
+
+def profile_end(capacity: int = 4096):
+    """-> list of (kernel name, milliseconds) in launch order."""
+    names = C.create_string_buffer(capacity * 32)
+    ms = (C.c_float * capacity)()
+    n = lib().vscan_profile_end(names, ms, capacity)
+    if n < 0:
+        raise VScanError(ERR_INVALID_ARG, "vscan_profile_end")
+    raw = names.raw
+    return [(raw[i * 32:(i + 1) * 32].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n)]
 
 
 def vscan_check(workspace: Workspace) -> int:

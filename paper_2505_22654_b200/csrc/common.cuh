@@ -34,6 +34,20 @@ inline vscan_status cuda_fail(cudaError_t e) {
     if (e__ != cudaSuccess) return ::vscan::cuda_fail(e__);    \
   } while (0)
 
+// Optional per-kernel timing (vscan_profile_begin / vscan_profile_end): when enabled, every launch
+// is bracketed by a pair of CUDA events on its stream.
+void prof_before(const char* name, cudaStream_t stream);
+void prof_after(cudaStream_t stream);
+
+// Launch wrapper: VSCAN_LAUNCH("name", stream, kernel<<<grid, block, smem, stream>>>(args));
+#define VSCAN_LAUNCH(name, stream, ...)        \
+  do {                                         \
+    ::vscan::prof_before(name, stream);        \
+    __VA_ARGS__;                               \
+    ::vscan::prof_after(stream);               \
+    VSCAN_AFTER_LAUNCH();                      \
+  } while (0)
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }

@@ -137,9 +137,8 @@ __global__ void __launch_bounds__(256) assign_simt_kernel(MergeParams p) {
 
 vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t stream) {
   dim3 grid((p.n_tokens + kTileT - 1) / kTileT, p.instances);
-  if (dtype == VSCAN_F32) assign_simt_kernel<float><<<grid, 256, 0, stream>>>(p);
-  else assign_simt_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(p);
-  VSCAN_AFTER_LAUNCH();
+  if (dtype == VSCAN_F32) VSCAN_LAUNCH("assign_simt", stream, assign_simt_kernel<float><<<grid, 256, 0, stream>>>(p));
+  else VSCAN_LAUNCH("assign_simt", stream, assign_simt_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(p));
   return VSCAN_OK;
 }
 
@@ -245,12 +244,11 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   dim3 grid((p.n_kept + kSlotsPerCta - 1) / kSlotsPerCta, p.instances);
   if (p.dim / E <= 128) {
     VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4>, smem));
-    group_mean_kernel<T, 4><<<grid, 256, smem, stream>>>(p);
+    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 4><<<grid, 256, smem, stream>>>(p)));
   } else {
     VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8>, smem));
-    group_mean_kernel<T, 8><<<grid, 256, smem, stream>>>(p);
+    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 8><<<grid, 256, smem, stream>>>(p)));
   }
-  VSCAN_AFTER_LAUNCH();
   return VSCAN_OK;
 }
 
@@ -330,9 +328,8 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   }
 
   dim3 ngrid((d->n_kept + 7) / 8, d->instances);
-  if (d->dtype == VSCAN_F32) kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p);
-  else kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p);
-  VSCAN_AFTER_LAUNCH();
+  if (d->dtype == VSCAN_F32) VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p));
+  else VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p));
 
   st = tensor ? launch_assign_tensor(p, stream) : launch_assign_simt(d->dtype, p, stream);
   if (st != VSCAN_OK) return st;

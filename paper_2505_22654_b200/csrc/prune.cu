@@ -200,9 +200,9 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
     const size_t smem = static_cast<size_t>(d->n_vis) * 4 + 16;
     VSCAN_CUDA_TRY(allow_smem(prune_topk_kernel, smem));
     const int threads = d->n_vis <= 2048 ? 256 : 1024;
-    prune_topk_kernel<<<d->batch, threads, smem, stream>>>(probs, d->scores, d->kept_vis, d->q_heads, d->n_vis,
-                                                           d->k_keep);
-    VSCAN_AFTER_LAUNCH();
+    VSCAN_LAUNCH("prune_topk", stream,
+                 prune_topk_kernel<<<d->batch, threads, smem, stream>>>(probs, d->scores, d->kept_vis, d->q_heads,
+                                                                        d->n_vis, d->k_keep));
   }
   if (seq_out == 0) return VSCAN_OK;
   const size_t e = dtype_bytes(d->dtype);
@@ -217,7 +217,6 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   c.hidden_vecs = d->hidden ? static_cast<int>(d->hidden_dim * e / 16) : 0;
   c.kv_vecs = static_cast<int>(d->head_dim * e / 16);
   dim3 grid(seq_out, d->batch);
-  compact_kernel<<<grid, kCompactThreads, 0, stream>>>(c);
-  VSCAN_AFTER_LAUNCH();
+  VSCAN_LAUNCH("compact", stream, compact_kernel<<<grid, kCompactThreads, 0, stream>>>(c));
   return VSCAN_OK;
 }

@@ -39,12 +39,11 @@ vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStre
   dim3 grid(p.q_heads, batch);
   if (dtype == VSCAN_F32) {
     VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<float>, smem));
-    qk_softmax_kernel<float><<<grid, 256, smem, stream>>>(p);
+    VSCAN_LAUNCH("qk_softmax", stream, qk_softmax_kernel<float><<<grid, 256, smem, stream>>>(p));
   } else {
     VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<__nv_bfloat16>, smem));
-    qk_softmax_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(p);
+    VSCAN_LAUNCH("qk_softmax", stream, qk_softmax_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(p));
   }
-  VSCAN_AFTER_LAUNCH();
   return VSCAN_OK;
 }
 
@@ -102,13 +101,14 @@ extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, 
     if (d->instances == 0 || d->n_tokens == 0) return VSCAN_OK;
     dim3 grid((d->n_tokens + 255) / 256, d->instances);
     if (d->dtype == VSCAN_F32)
-      row_mean_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(d->attn), d->scores, d->heads,
-                                                       d->row_len, d->cls_offset, d->n_tokens);
+      VSCAN_LAUNCH("row_mean", stream,
+                   row_mean_kernel<float><<<grid, 256, 0, stream>>>(static_cast<const float*>(d->attn), d->scores,
+                                                                    d->heads, d->row_len, d->cls_offset, d->n_tokens));
     else
-      row_mean_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(d->attn),
-                                                               d->scores, d->heads, d->row_len, d->cls_offset,
-                                                               d->n_tokens);
-    VSCAN_AFTER_LAUNCH();
+      VSCAN_LAUNCH("row_mean", stream,
+                   row_mean_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
+                       static_cast<const __nv_bfloat16*>(d->attn), d->scores, d->heads, d->row_len, d->cls_offset,
+                       d->n_tokens));
     return VSCAN_OK;
   }
   if (d->batch == 0 || d->span_len == 0) return VSCAN_OK;
@@ -125,7 +125,6 @@ extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, 
   st = launch_qk_softmax(d->dtype, p, d->batch, stream);
   if (st != VSCAN_OK) return st;
   dim3 grid((d->span_len + 255) / 256, d->batch);
-  head_mean_kernel<<<grid, 256, 0, stream>>>(p.probs, d->scores, d->q_heads, d->span_len);
-  VSCAN_AFTER_LAUNCH();
+  VSCAN_LAUNCH("head_mean", stream, head_mean_kernel<<<grid, 256, 0, stream>>>(p.probs, d->scores, d->q_heads, d->span_len));
   return VSCAN_OK;
 }

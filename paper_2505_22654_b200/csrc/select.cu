@@ -128,7 +128,7 @@ extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, vo
   const size_t smem = static_cast<size_t>(n) * 9 + 16;
   VSCAN_CUDA_TRY(allow_smem(select_kernel, smem));
   const int threads = n <= 2048 ? 256 : 1024;
-  select_kernel<<<d->instances, threads, smem, static_cast<cudaStream_t>(stream)>>>(p);
-  VSCAN_AFTER_LAUNCH();
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  VSCAN_LAUNCH("select", st, select_kernel<<<d->instances, threads, smem, st>>>(p));
   return VSCAN_OK;
 }
