@@ -100,6 +100,31 @@ vscan_status vscan_score(const vscan_score_desc* desc, void* workspace, size_t w
                          void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * vscan_score_qk_static  (the paper has no counterpart: this is a packaging variant of the QK mode
+ * above, same arithmetic, same result)
+ *
+ * For callers that cannot allocate device memory and therefore have no workspace to pass: code that
+ * runs inside someone else's memory plan (an inference server whose pool is sized and frozen at
+ * start-up, a plugin that is handed tensors but no allocator), or inside a region where
+ * cudaMalloc is forbidden or would stall everything else on the GPU.  The call takes only the inputs
+ * and the output; its scratch (the per-head probabilities, batch * q_heads * span_len floats) is a
+ * fixed array built into the library, vscan_score_qk_static_capacity() floats long (1 Mi floats =
+ * 4 MiB).  Every GPU on which the library is loaded carries those 4 MiB until the process exits.
+ * The function calls no allocator of any kind.
+ *   desc    a vscan_score_desc with mode = VSCAN_SCORE_QK; the fields mean what they mean above.
+ *   Returns VSCAN_ERR_UNSUPPORTED when batch * q_heads * span_len exceeds the capacity (nothing is
+ *   launched); the other statuses as for vscan_score.
+ * The first call on a given device looks up the array's device address (one runtime query, cached per
+ * device); make that first call outside any stream capture, with the target device current.
+ * All calls on one GPU share the one array and it keeps whatever the last call left there.  A call
+ * overwrites every entry it later reads, so stale contents are harmless and nothing needs clearing,
+ * but two calls whose kernels overlap in time on the same GPU (different streams, or different host
+ * threads) race on it and give wrong scores: keep calls on one stream, or order them yourself.
+ * ------------------------------------------------------------------------------------------- */
+size_t vscan_score_qk_static_capacity(void);
+vscan_status vscan_score_qk_static(const vscan_score_desc* desc, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * vscan_select_global_local (Sec. 4.1, Eq. 2-3 and the footnote on duplicates)
  *
  * Tokens of an instance are numbered t = f*grid_h*grid_w + r*grid_w + c.  The grid is cut into

@@ -85,6 +85,9 @@ def lib() -> C.CDLL:
         L.vscan_profile_begin.restype, L.vscan_profile_begin.argtypes = _i32, [_i32]
         L.vscan_profile_end.restype = _i32
         L.vscan_profile_end.argtypes = [C.c_char_p, C.POINTER(C.c_float), _i32]
+        L.vscan_score_qk_static_capacity.restype = C.c_size_t
+        L.vscan_score_qk_static.restype = _i32
+        L.vscan_score_qk_static.argtypes = [C.POINTER(ScoreDesc), _vp]
         _LIB = L
     return _LIB
 
@@ -186,6 +189,19 @@ def vscan_score_qk(q, k, span_begin, span_len, scale, softmax_span=SPAN_ONLY, ou
         out = torch.empty((q.shape[0], span_len), dtype=torch.float32, device=q.device)
     d = score_qk_desc(q, k, span_begin, span_len, scale, softmax_span, out)
     _call("vscan_score", d, "vscan_score_workspace_bytes", workspace)
+    return out
+
+
+def vscan_score_qk_static(q, k, span_begin, span_len, scale, out, softmax_span=SPAN_ONLY):
+    """Same scores as vscan_score_qk, for callers that may not allocate device memory: the scratch
+    is a fixed 4 MiB array inside the library instead of a workspace, and nothing is allocated here
+    either, so the caller brings `out` ([B, span_len] float32).  Raises VScanError(ERR_UNSUPPORTED)
+    when B * Hq * span_len exceeds the built-in capacity.  Calls on one GPU share the scratch: do not
+    let two of them overlap."""
+    d = score_qk_desc(q, k, span_begin, span_len, scale, softmax_span, out)
+    st = lib().vscan_score_qk_static(C.byref(d), _stream())
+    if st != OK:
+        raise VScanError(st, "vscan_score_qk_static")
     return out
 
 
