@@ -331,7 +331,14 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   if (d->dtype == VSCAN_F32) VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p));
   else VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p));
 
-  st = tensor ? launch_assign_tensor(p, stream) : launch_assign_simt(d->dtype, p, stream);
+  if (tensor) {
+    st = launch_assign_tensor(p, stream);
+    // a shape the tensor path cannot take (tensor-map limits) runs on the CUDA cores unless the
+    // caller insisted on tensor cores
+    if (st == VSCAN_ERR_UNSUPPORTED && d->path == VSCAN_MERGE_AUTO) st = launch_assign_simt(d->dtype, p, stream);
+  } else {
+    st = launch_assign_simt(d->dtype, p, stream);
+  }
   if (st != VSCAN_OK) return st;
 
   return d->dtype == VSCAN_F32 ? launch_group_mean<float>(p, stream)

@@ -139,6 +139,35 @@ def test_merge_exact_ties_and_duplicates():
     assert int(a2[0, 4]) == 0
 
 
+@pytest.mark.parametrize("N,D,K1,c", [(576, 1024, 64, 1), (576, 1024, 192, 1), (300, 72, 17, 0), (130, 264, 130, 1),
+                                      (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0)])
+def test_merge_tensor_path_matches_oracle(N, D, K1, c):
+    """The tcgen05 path on its own (path = TENSOR): tile tails, kept counts that are not multiples of
+    16, more than 256 kept tokens (several accumulator rounds), feature dims that are not multiples
+    of 64."""
+    cfg = small_cfg("bf16", grid_h=1, grid_w=N, win_h=1, win_w=N, k_w=0, k_g=K1, D=D, C=1, B=2, cls=c)
+    x = round_to_dtype(RNG.standard_normal((2, N + c, D)).astype(np.float32), "bf16")
+    kept = np.stack([np.sort(RNG.choice(N, K1, replace=False)) for _ in range(2)])
+    plant.plant_merge(cfg, x, kept)
+    ws = vs.Workspace(1 << 20)
+    merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
+                                            want_counts=True, path=vs.MERGE_TENSOR, workspace=ws)
+    assert vs.vscan_check(ws) == 0
+    for b in range(2):
+        m, a, cn = vo.merge(x[b], c, kept[b])
+        np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
+        np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
+        check_merged(merged[b], m, "bf16")
+
+
+def test_merge_tensor_path_refuses_fp32():
+    x = torch.randn((1, 40, 16), device="cuda")
+    kept = torch.tensor([[1, 5]], dtype=torch.int32, device="cuda")
+    with pytest.raises(vs.VScanError) as e:
+        vs.vscan_merge(x, 0, kept, path=vs.MERGE_TENSOR)
+    assert e.value.status == 2
+
+
 def test_merge_separate_metric():
     x = RNG.standard_normal((2, 50, 24)).astype(np.float32)
     metric = RNG.standard_normal((2, 50, 16)).astype(np.float32)
