@@ -1,11 +1,12 @@
 // Tensor-core path of the merge assignment (Sec. 4.1 "Token Merging"): for a tile of 128 tokens the
 // dot products with all kept tokens are one tcgen05 MMA chain, D[128 x Nk] (fp32, tensor memory) =
 // A[128 tokens x dim] * B[Nk kept x dim]^T with bf16 operands in shared memory.
-//   warp 0      TMA producer of the token tile (3-D tensor map over [instance][row][dim], 128B swizzle)
+//   warp 0      TMA producer: the token tile (3-D tensor map over [instance][row][dim], 128B swizzle) and
+//               the kept rows, which are not contiguous, four rows per TMA gather
 //   warp 1      allocates tensor memory, issues the MMAs (one elected lane), commits to mbarriers
-//   warps 2-5   gather the kept rows into the swizzled B stage (kept rows are not contiguous), then
-//               read the accumulator back (tcgen05.ld, one token row per thread), scale by 1/|m_s|
-//               and keep the running arg-max (lowest slot on ties)
+//   warps 2-5   read the accumulator back (tcgen05.ld, one token row per thread), scale by 1/|m_s|
+//               and keep the running arg-max (lowest slot on ties); with more than 256 kept tokens
+//               two accumulators alternate so this overlaps the next round of MMAs
 // The similarity matrix never leaves the SM.  Every mbarrier wait is bounded: on expiry the CTA
 // records VSCAN_ERR_TIMEOUT in the status word, lets copies in flight land, frees its tensor memory
 // and returns.
@@ -81,6 +82,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       : "memory");
 }
 
+// Four rows of a 2-D tensor (box = one row of 64 elements) land as four consecutive 128-byte rows.
+__device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* map, uint64_t* bar, int col, int r0, int r1,
+                                            int r2, int r3) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(col), "r"(r0), "r"(r1),
+        "r"(r2), "r"(r3)
+      : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr) {
   uint64_t d = 0;
@@ -132,19 +144,19 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* v) {
 }
 
 struct Shared {
-  uint64_t full[kMaxStages];    // A landed (tx bytes) and B gathered (4 warp arrivals)
+  uint64_t full[kMaxStages];    // token tile and kept rows of the stage have landed (transaction bytes)
   uint64_t empty[kMaxStages];   // MMAs that read the stage have completed
-  uint64_t tmem_full;           // accumulator of the current n-chunk complete
-  uint64_t tmem_empty;          // epilogue has read the accumulator
+  uint64_t tmem_full[2];        // accumulator (ping or pong) of an n-chunk complete
+  uint64_t tmem_empty[2];       // epilogue has read that accumulator
   uint32_t tmem_base;
   int abort_flag;
   int best_slot[kTileM];
-  float inv_norm[kMaxN];
-  int kept_row[kMaxN];
+  float inv_norm[2][kMaxN];
 };
 
 // dynamic shared memory (1024-byte aligned): stages x [A tile 128x64 bf16 | B tile n_pad x 64 bf16]
-__global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_constant__ CUtensorMap map_a, Params p) {
+__global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                 const __grid_constant__ CUtensorMap map_b, Params p) {
   extern __shared__ unsigned char smem_dyn[];
   __shared__ Shared sh;
   // the swizzle pattern is a function of the shared-memory address: stage bases sit on 1024 bytes
@@ -154,11 +166,11 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
   const MergeParams& m = p.m;
   volatile int* abort_flag = &sh.abort_flag;
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 5); mbar_init(&sh.empty[s], 1); }
-    mbar_init(&sh.tmem_full, 1);
-    mbar_init(&sh.tmem_empty, 4);
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 4); }
     sh.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -172,15 +184,41 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
   const uint32_t tmem_acc = sh.tmem_base;
 
   if (warp == 0) {
-    // ------------------------------------------------------------ token tile producer (TMA)
-    if (lane == 0) {
-      int it = 0;
-      for (int nc = 0; nc < p.n_chunks && !*abort_flag; ++nc) {
-        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-          const int s = it % p.stages, round = it / p.stages;
-          if (round > 0 && !mbar_wait(&sh.empty[s], (round - 1) & 1, abort_flag)) break;
-          mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes);
-          tma_load_3d(tiles + s * stage_bytes, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
+    // ------------------------------------------------------------ producer: TMA tile + TMA row gathers
+    // Lane l issues the gathers of row groups l, l+32, ... (four kept rows each); it keeps their row
+    // coordinates in registers for the whole n-chunk.  Padding rows repeat the first kept row (their
+    // columns are masked in the epilogue).
+    const int groups = p.n_pad / 4;                 // gathers per stage
+    const int row_base = b * m.row_len + m.cls_offset;
+    const int first = row_base + min(max(kept[0], 0), m.n_tokens - 1);
+    int it = 0;
+    bool ok = true;
+    for (int nc = 0; nc < p.n_chunks; ++nc) {
+      int rows[2][4];
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int g = lane + 32 * i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int s_idx = nc * p.n_pad + g * 4 + j;
+          rows[i][j] = (g < groups && s_idx < m.n_kept) ? row_base + min(max(kept[s_idx], 0), m.n_tokens - 1) : first;
+        }
+      }
+      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+        const int s = it % p.stages, round = it / p.stages;
+        if (ok && round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
+        if (!ok) continue;
+        unsigned char* at = tiles + s * stage_bytes;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes + p.n_pad * 128);
+          tma_load_3d(at, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int g = lane + 32 * i;
+          if (g < groups)
+            tma_gather4(at + p.a_stage_bytes + g * 512, &map_b, &sh.full[s], kc * kChunkK, rows[i][0], rows[i][1],
+                        rows[i][2], rows[i][3]);
         }
       }
     }
@@ -190,10 +228,12 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
       const uint32_t idesc = instr_desc_bf16(p.n_pad);
       int it = 0;
       for (int nc = 0; nc < p.n_chunks && !*abort_flag; ++nc) {
-        if (nc > 0) {
-          if (!mbar_wait(&sh.tmem_empty, (nc - 1) & 1, abort_flag)) break;
+        const int acc = nc & 1, use = nc >> 1;
+        if (use > 0) {
+          if (!mbar_wait(&sh.tmem_empty[acc], (use - 1) & 1, abort_flag)) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         }
+        const uint32_t d_addr = tmem_acc + acc * p.n_pad;
         bool ok = true;
         for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
           const int s = it % p.stages, round = it / p.stages;
@@ -203,74 +243,35 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
           const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
 #pragma unroll
           for (int k = 0; k < kChunkK / 16; ++k)   // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
-            umma_bf16(tmem_acc, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
+            umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
           umma_commit(&sh.empty[s]);
         }
         if (!ok) break;
-        umma_commit(&sh.tmem_full);
+        umma_commit(&sh.tmem_full[acc]);
       }
     }
   } else {
-    // ------------------------------------------------------------ kept-row gather, then epilogue
-    const int pw = warp - 2;                  // 0..3
-    const int ptid = pw * 32 + lane;          // 0..127
+    // ------------------------------------------------------------ epilogue: accumulator -> arg-max
+    const int ptid = (warp - 2) * 32 + lane;  // 0..127
     const int quarter = warp & 3;             // tensor-memory lanes this warp may read
     const int row = quarter * 32 + lane;      // token row of this thread within the tile
-    const __nv_bfloat16* mb = static_cast<const __nv_bfloat16*>(m.metric) +
-                              (static_cast<size_t>(b) * m.row_len + m.cls_offset) * m.metric_dim;
-    const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
     float best_val = -INFINITY;
     int best_idx = 0;
-    int it = 0;
     bool ok = true;
-    // Once `ok` drops the loops keep running with their work skipped, so that the four warps execute
+    // Once `ok` drops the loop keeps running with its work skipped, so that the four warps execute
     // the same sequence of named barriers and warp-wide instructions whatever happens.
     for (int nc = 0; nc < p.n_chunks; ++nc) {
-      const int n0 = nc * p.n_pad;
-      // stage the kept rows and scales of this n-chunk (only these four warps touch them)
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const int n0 = nc * p.n_pad, acc = nc & 1, use = nc >> 1;
+      // scales of this n-chunk; the buffer was last read two chunks ago, before that chunk's arrive
       for (int j = ptid; j < p.n_pad; j += 128) {
         const int s_idx = n0 + j;
-        sh.kept_row[j] = s_idx < m.n_kept ? min(max(kept[s_idx], 0), m.n_tokens - 1) : -1;
-        sh.inv_norm[j] = s_idx < m.n_kept ? m.inv_norm[static_cast<size_t>(b) * m.n_kept + s_idx] : 0.f;
+        sh.inv_norm[acc][j] = s_idx < m.n_kept ? m.inv_norm[static_cast<size_t>(b) * m.n_kept + s_idx] : 0.f;
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      const int chunks = p.n_pad * 8;          // 16-byte pieces per B stage
-      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-        const int s = it % p.stages, round = it / p.stages;
-        if (ok && round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
-        if (!ok) continue;
-        unsigned char* bt = tiles + s * stage_bytes + p.a_stage_bytes;
-        const int col0 = kc * kChunkK;
-        for (int c0 = ptid; c0 < chunks; c0 += 128 * 4) {
-          uint4 v[4];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int c = c0 + u * 128;
-            v[u] = make_uint4(0u, 0u, 0u, 0u);
-            if (c < chunks) {
-              const int r = c >> 3, piece = c & 7, tk = sh.kept_row[r], col = col0 + piece * 8;
-              if (tk >= 0 && col < m.metric_dim) v[u] = ld_nc_16(mb + static_cast<size_t>(tk) * m.metric_dim + col);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int c = c0 + u * 128;
-            if (c < chunks) {
-              const int r = c >> 3, piece = c & 7;
-              *reinterpret_cast<uint4*>(bt + r * 128 + ((piece ^ (r & 7)) << 4)) = v[u];
-            }
-          }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the stores visible to the MMA
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.full[s]);
-      }
-      // accumulator of this n-chunk -> running arg-max of this thread's token row
-      if (ok) ok = mbar_wait_warp(&sh.tmem_full, nc & 1, abort_flag);
+      if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
       if (!ok) continue;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16);
+      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.n_pad;
       for (int c0 = 0; c0 < p.n_pad; c0 += 32) {
         uint32_t v[32];
         if (p.n_pad - c0 >= 32) tmem_ld32(taddr + c0, v);
@@ -284,14 +285,14 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
         for (int j = 0; j < 32; ++j) {
           const int s_idx = n0 + c0 + j;
           if (c0 + j < p.n_pad && s_idx < m.n_kept) {
-            const float val = __uint_as_float(v[j]) * sh.inv_norm[c0 + j];
+            const float val = __uint_as_float(v[j]) * sh.inv_norm[acc][c0 + j];
             if (val > best_val) { best_val = val; best_idx = s_idx; }
           }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(&sh.tmem_empty);
+      if (lane == 0) mbar_arrive(&sh.tmem_empty[acc]);
     }
     sh.best_slot[row] = best_idx;
     asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -344,8 +345,8 @@ static bool plan(const MergeParams& m, Params& p) {
   p.n_pad = n16 <= kMaxN ? n16 : kMaxN;
   p.n_chunks = (m.n_kept + p.n_pad - 1) / p.n_pad;
   p.k_chunks = (m.metric_dim + kChunkK - 1) / kChunkK;
-  p.tmem_cols = 32;
-  while (p.tmem_cols < p.n_pad) p.tmem_cols *= 2;
+  p.tmem_cols = 32;   // one accumulator, or two (ping-pong) when the kept set needs several rounds
+  while (p.tmem_cols < p.n_pad * (p.n_chunks > 1 ? 2 : 1)) p.tmem_cols *= 2;
   p.a_stage_bytes = kTileM * kChunkK * 2;
   p.b_stage_bytes = ((p.n_pad * kChunkK * 2) + 1023) / 1024 * 1024;
   const int stage = p.a_stage_bytes + p.b_stage_bytes;
@@ -383,10 +384,20 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
                       elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
+  // kept rows: the same memory as a 2-D [all rows][dim] tensor, fetched four rows at a time
+  CUtensorMap map_b;
+  const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(m.metric_dim),
+                                static_cast<cuuint64_t>(m.row_len) * static_cast<cuuint64_t>(m.instances)};
+  const cuuint64_t strides_b[1] = {static_cast<cuuint64_t>(m.metric_dim) * 2};
+  const cuuint32_t box_b[2] = {tc::kChunkK, 1};
+  r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(m.metric), dims_b, strides_b, box_b, elem,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
   const size_t smem = static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
   dim3 grid((m.n_tokens + tc::kTileM - 1) / tc::kTileM, m.instances);
-  VSCAN_LAUNCH("assign_tensor", stream, tc::assign_tensor_kernel<<<grid, tc::kThreads, smem, stream>>>(map, p));
+  VSCAN_LAUNCH("assign_tensor", stream, tc::assign_tensor_kernel<<<grid, tc::kThreads, smem, stream>>>(map, map_b, p));
   return VSCAN_OK;
 }
 
