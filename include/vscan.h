@@ -152,6 +152,25 @@ vscan_status vscan_select_global_local(const vscan_select_desc* desc, void* work
                                        size_t workspace_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * vscan_score_select (Eq. 2 and Eq. 3 in one launch)
+ *
+ * The same result as two ROW-mode vscan_score calls followed by vscan_select_global_local, without
+ * the scores going through memory: the head means of attn_global / attn_local (layouts and meaning as
+ * in vscan_score, ROW mode; the two may be the same buffer) are taken inside the selection kernel.
+ *   select.scores_global / select.scores_local are here OPTIONAL OUTPUTS ([instances][N] float32)
+ *   that receive the head means; every other field of `select` means what it means above.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t dtype; /* vscan_dtype of the attention rows */
+  const void* attn_global;
+  const void* attn_local;
+  int32_t heads, row_len, cls_offset;
+  vscan_select_desc select;
+} vscan_score_select_desc;
+
+vscan_status vscan_score_select(const vscan_score_select_desc* desc, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * vscan_merge (Sec. 4.1 "Token Merging", Eq. 4)
  *
  * For every token u not in kept_idx: a(u) = argmax_s cos(m_u, m_kept[s]) (lowest slot on ties; norms

@@ -36,6 +36,11 @@ class SelectDesc(C.Structure):
                 ("k_per_window", _i32), ("k_global", _i32), ("kept_idx", _vp), ("kept_mask", _vp)]
 
 
+class ScoreSelectDesc(C.Structure):
+    _fields_ = [("dtype", _i32), ("attn_global", _vp), ("attn_local", _vp), ("heads", _i32), ("row_len", _i32),
+                ("cls_offset", _i32), ("select", SelectDesc)]
+
+
 class MergeDesc(C.Structure):
     _fields_ = [("dtype", _i32), ("path", _i32), ("x", _vp), ("metric", _vp), ("kept_idx", _vp),
                 ("instances", _i32), ("row_len", _i32), ("cls_offset", _i32), ("n_tokens", _i32),
@@ -77,6 +82,8 @@ def lib() -> C.CDLL:
                          ("vscan_merge", MergeDesc), ("vscan_llm_prune", PruneDesc)):
             f = getattr(L, fn)
             f.restype, f.argtypes = _i32, [C.POINTER(desc), _vp, C.c_size_t, _vp]
+        L.vscan_score_select.restype = _i32
+        L.vscan_score_select.argtypes = [C.POINTER(ScoreSelectDesc), _vp]
         L.vscan_version.restype = _i32
         L.vscan_status_string.restype, L.vscan_status_string.argtypes = C.c_char_p, [_i32]
         L.vscan_check.restype, L.vscan_check.argtypes = _i32, [_vp, _vp]
@@ -221,6 +228,26 @@ def vscan_select_global_local(scores_global, scores_local, frames, grid_h, grid_
     if st != OK:
         raise VScanError(st, "vscan_select_global_local")
     return (out, mask) if want_mask else out
+
+
+def vscan_score_select(attn_global, attn_local, cls_offset, frames, grid_h, grid_w, win_h, win_w, k_per_window,
+                       k_global, out=None, scores_global=None, scores_local=None):
+    """Eq. 2 + Eq. 3 in one launch: head means of the two attention tensors and the selection.
+    -> kept_idx [B', K1] int32.  scores_global / scores_local, if given, receive the head means."""
+    B, H, L = attn_global.shape
+    windows = frames * (grid_h // max(win_h, 1)) * (grid_w // max(win_w, 1))
+    k1 = windows * k_per_window + k_global
+    if out is None:
+        out = torch.empty((B, max(k1, 0)), dtype=torch.int32, device=attn_global.device)
+    sd = SelectDesc(scores_global=_ptr(scores_global), scores_local=_ptr(scores_local), instances=B, frames=frames,
+                    grid_h=grid_h, grid_w=grid_w, win_h=win_h, win_w=win_w, k_per_window=k_per_window,
+                    k_global=k_global, kept_idx=_ptr(out), kept_mask=None)
+    d = ScoreSelectDesc(dtype=_dtype_code(attn_global), attn_global=_ptr(attn_global), attn_local=_ptr(attn_local),
+                        heads=H, row_len=L, cls_offset=cls_offset, select=sd)
+    st = lib().vscan_score_select(C.byref(d), _stream())
+    if st != OK:
+        raise VScanError(st, "vscan_score_select")
+    return out
 
 
 def vscan_merge(x, cls_offset, kept_idx, n_tokens=None, metric=None, path=MERGE_AUTO, out=None,

@@ -5,46 +5,6 @@
 
 namespace vscan {
 
-// One CTA per sequence: head mean (h ascending), radix select, ascending survivor list.
-// dynamic shared memory: keys[n_vis]
-__global__ void __launch_bounds__(1024) prune_topk_kernel(const float* __restrict__ probs, float* scores_out,
-                                                          int32_t* kept_vis, int q_heads, int n_vis, int k_keep) {
-  extern __shared__ __align__(16) uint32_t keys[];
-  __shared__ SelectScratch sc;
-  const int b = blockIdx.x;
-  const float* base = probs + static_cast<size_t>(b) * q_heads * n_vis;
-  for (int j = threadIdx.x; j < n_vis; j += blockDim.x) {
-    float acc = 0.f;
-    for (int h = 0; h < q_heads; ++h) acc += base[static_cast<size_t>(h) * n_vis + j];
-    acc /= static_cast<float>(q_heads);
-    if (scores_out) scores_out[static_cast<size_t>(b) * n_vis + j] = acc;
-    keys[j] = float_to_key(acc);
-  }
-  __syncthreads();
-  if (k_keep <= 0) return;
-  uint32_t thr;
-  int need;
-  block_radix_select(keys, nullptr, n_vis, k_keep, sc, thr, need);
-  const int per = (n_vis + blockDim.x - 1) / blockDim.x;
-  const int lo = min(n_vis, static_cast<int>(threadIdx.x) * per), hi = min(n_vis, lo + per);
-  int eq_local = 0;
-  for (int i = lo; i < hi; ++i) eq_local += (keys[i] == thr);
-  int total;
-  int eq_before = block_exclusive_scan(eq_local, sc.warp_sums, total);
-  int kept_local = 0;
-  unsigned long long flags = 0;  // per <= 64 because n_vis <= 16384 and blockDim >= 256
-  for (int i = lo; i < hi; ++i) {
-    uint32_t key = keys[i];
-    bool keep = key > thr;
-    if (key == thr) { keep = eq_before < need; ++eq_before; }
-    if (keep) { flags |= 1ull << (i - lo); ++kept_local; }
-  }
-  int pos = block_exclusive_scan(kept_local, sc.warp_sums, total);
-  int32_t* out = kept_vis + static_cast<size_t>(b) * k_keep;
-  for (int i = lo; i < hi; ++i)
-    if ((flags >> (i - lo)) & 1ull) { if (pos < k_keep) out[pos] = i; ++pos; }
-}
-
 struct CompactParams {
   const int32_t* kept_vis;  // [batch][k_keep]
   const uint4* hidden; uint4* hidden_out;
@@ -173,7 +133,8 @@ static vscan_status validate_prune(const vscan_prune_desc* d) {
 
 extern "C" size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* d) {
   if (!d || d->batch <= 0 || d->q_heads <= 0 || d->n_vis <= 0) return kStatusBytes;
-  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * d->q_heads * d->n_vis * sizeof(float), 256);
+  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * sizeof(int), 256) +
+         round_up(static_cast<size_t>(d->batch) * d->q_heads * d->n_vis * sizeof(float), 256);
 }
 
 extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspace, size_t workspace_bytes,
@@ -186,23 +147,26 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   const size_t need = vscan_llm_prune_workspace_bytes(d);
   if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
   const int seq_len = d->n_sys + d->n_vis + d->n_txt, seq_out = seq_len - d->n_vis + d->k_keep;
-  float* probs = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+  // workspace: status word | per-sequence arrival counters | per-head probabilities
+  char* ws = static_cast<char*>(workspace);
+  const size_t counter_bytes = round_up(static_cast<size_t>(d->batch) * sizeof(int), 256);
 
   if (d->n_vis > 0) {
     QkParams p;
-    p.q = d->q_last; p.k = d->k; p.probs = probs; p.status = static_cast<uint32_t*>(workspace);
+    p.q = d->q_last; p.k = d->k; p.status = static_cast<uint32_t*>(workspace);
+    p.counters = reinterpret_cast<int*>(ws + kStatusBytes);
+    p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes);
+    p.scores = d->scores; p.kept = d->kept_vis; p.k_keep = d->k_keep;
     p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = seq_len; p.head_dim = d->head_dim;
     p.span_begin = d->n_sys; p.span_len = d->n_vis; p.scale = d->scale;
     if (d->softmax_span == VSCAN_SPAN_ONLY) { p.soft_lo = d->n_sys; p.soft_n = d->n_vis; }
     else { p.soft_lo = 0; p.soft_n = seq_len; }
+    // score and top-k in one launch: the last CTA of each sequence reduces over the heads and selects
+    VSCAN_CUDA_TRY(cudaMemsetAsync(p.counters, 0, counter_bytes, stream));
     st = launch_qk_softmax(d->dtype, p, d->batch, stream);
     if (st != VSCAN_OK) return st;
-    const size_t smem = static_cast<size_t>(d->n_vis) * 4 + 16;
-    VSCAN_CUDA_TRY(allow_smem(prune_topk_kernel, smem));
-    const int threads = d->n_vis <= 2048 ? 256 : 1024;
-    VSCAN_LAUNCH("prune_topk", stream,
-                 prune_topk_kernel<<<d->batch, threads, smem, stream>>>(probs, d->scores, d->kept_vis, d->q_heads,
-                                                                        d->n_vis, d->k_keep));
+  } else {
+    VSCAN_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, stream));
   }
   if (seq_out == 0) return VSCAN_OK;
   const size_t e = dtype_bytes(d->dtype);

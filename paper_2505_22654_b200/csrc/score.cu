@@ -12,39 +12,41 @@ __global__ void __launch_bounds__(256) row_mean_kernel(const T* __restrict__ att
   const T* base = attn + static_cast<size_t>(blockIdx.y) * heads * row_len + cls_offset + j;
   float acc = 0.f;
   int h = 0;
-  for (; h + 4 <= heads; h += 4) {
-    float a0 = to_float(base[static_cast<size_t>(h) * row_len]);
-    float a1 = to_float(base[static_cast<size_t>(h + 1) * row_len]);
-    float a2 = to_float(base[static_cast<size_t>(h + 2) * row_len]);
-    float a3 = to_float(base[static_cast<size_t>(h + 3) * row_len]);
-    acc += a0; acc += a1; acc += a2; acc += a3;
+  for (; h + 8 <= heads; h += 8) {   // eight independent loads in flight, added in head order
+    float a[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) a[u] = to_float(base[static_cast<size_t>(h + u) * row_len]);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += a[u];
   }
   for (; h < heads; ++h) acc += to_float(base[static_cast<size_t>(h) * row_len]);
   scores[static_cast<size_t>(blockIdx.y) * n_tokens + j] = acc / static_cast<float>(heads);
 }
 
-__global__ void head_mean_kernel(const float* __restrict__ probs, float* __restrict__ scores, int q_heads,
-                                 int span_len) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= span_len) return;
-  const float* base = probs + static_cast<size_t>(blockIdx.y) * q_heads * span_len + j;
-  float acc = 0.f;
-  for (int h = 0; h < q_heads; ++h) acc += base[static_cast<size_t>(h) * span_len];
-  scores[static_cast<size_t>(blockIdx.y) * span_len + j] = acc / static_cast<float>(q_heads);
+template <typename T>
+static vscan_status launch_qk_typed(const QkParams& p, int batch, size_t smem, cudaStream_t stream) {
+  constexpr int E = Vec16<T>::kElems;
+  dim3 grid(p.q_heads, batch);
+  const int vecs = p.head_dim / E;
+#define VSCAN_QK_CASE(VPS)                                                                          \
+  do {                                                                                              \
+    VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<T, VPS>, smem));                                    \
+    VSCAN_LAUNCH("qk_softmax", stream, (qk_softmax_kernel<T, VPS><<<grid, 256, smem, stream>>>(p))); \
+    return VSCAN_OK;                                                                                \
+  } while (0)
+  if (vecs == 16) VSCAN_QK_CASE(2);
+  if (vecs == 32) VSCAN_QK_CASE(4);
+  if (vecs == 8) VSCAN_QK_CASE(1);
+  VSCAN_QK_CASE(0);
+#undef VSCAN_QK_CASE
 }
 
 vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStream_t stream) {
   const size_t smem = qk_smem_bytes(p.head_dim, p.soft_n);
   if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
-  dim3 grid(p.q_heads, batch);
-  if (dtype == VSCAN_F32) {
-    VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<float>, smem));
-    VSCAN_LAUNCH("qk_softmax", stream, qk_softmax_kernel<float><<<grid, 256, smem, stream>>>(p));
-  } else {
-    VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<__nv_bfloat16>, smem));
-    VSCAN_LAUNCH("qk_softmax", stream, qk_softmax_kernel<__nv_bfloat16><<<grid, 256, smem, stream>>>(p));
-  }
-  return VSCAN_OK;
+  if (batch > 65535) return VSCAN_ERR_UNSUPPORTED;
+  return dtype == VSCAN_F32 ? launch_qk_typed<float>(p, batch, smem, stream)
+                            : launch_qk_typed<__nv_bfloat16>(p, batch, smem, stream);
 }
 
 }  // namespace vscan
@@ -87,7 +89,8 @@ static vscan_status validate_score(const vscan_score_desc* d) {
 
 extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
   if (!d || d->mode != VSCAN_SCORE_QK || d->batch <= 0 || d->q_heads <= 0 || d->span_len <= 0) return 0;
-  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * d->q_heads * d->span_len * sizeof(float), 256);
+  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * sizeof(int), 256) +
+         round_up(static_cast<size_t>(d->batch) * d->q_heads * d->span_len * sizeof(float), 256);
 }
 
 extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, size_t workspace_bytes,
@@ -114,17 +117,21 @@ extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, 
   if (d->batch == 0 || d->span_len == 0) return VSCAN_OK;
   const size_t need = vscan_score_workspace_bytes(d);
   if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
+  // workspace: status word | per-sequence arrival counters | per-head probabilities
+  char* ws = static_cast<char*>(workspace);
+  const size_t counter_bytes = round_up(static_cast<size_t>(d->batch) * sizeof(int), 256);
   QkParams p;
   p.q = d->q; p.k = d->k;
   p.status = static_cast<uint32_t*>(workspace);
-  p.probs = reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes);
+  p.counters = reinterpret_cast<int*>(ws + kStatusBytes);
+  p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes);
+  p.scores = d->scores;
   p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = d->seq_len; p.head_dim = d->head_dim;
   p.span_begin = d->span_begin; p.span_len = d->span_len; p.scale = d->scale;
   if (d->softmax_span == VSCAN_SPAN_ONLY) { p.soft_lo = d->span_begin; p.soft_n = d->span_len; }
   else { p.soft_lo = 0; p.soft_n = d->seq_len; }
+  VSCAN_CUDA_TRY(cudaMemsetAsync(p.counters, 0, counter_bytes, stream));
   st = launch_qk_softmax(d->dtype, p, d->batch, stream);
   if (st != VSCAN_OK) return st;
-  dim3 grid((d->span_len + 255) / 256, d->batch);
-  VSCAN_LAUNCH("head_mean", stream, head_mean_kernel<<<grid, 256, 0, stream>>>(p.probs, d->scores, d->q_heads, d->span_len));
   return VSCAN_OK;
 }

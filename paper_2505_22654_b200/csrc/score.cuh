@@ -2,28 +2,41 @@
 #pragma once
 
 #include "common.cuh"
+#include "topk.cuh"
 
 namespace vscan {
 
 struct QkParams {
-  const void* q;     // [batch][q_heads][head_dim]
-  const void* k;     // [batch][kv_heads][seq_len][head_dim]
-  float* probs;      // [batch][q_heads][span_len]  per-head probabilities on the span (workspace)
-  uint32_t* status;  // device status word of the workspace, cleared by the first CTA
-  int q_heads, kv_heads, seq_len, head_dim, span_begin, span_len;
-  int soft_lo, soft_n;  // keys the softmax runs over: [soft_lo, soft_lo + soft_n)
-  float scale;
+  const void* q = nullptr;     // [batch][q_heads][head_dim]
+  const void* k = nullptr;     // [batch][kv_heads][seq_len][head_dim]
+  float* probs = nullptr;      // [batch][q_heads][span_len]  per-head probabilities on the span (scratch)
+  uint32_t* status = nullptr;  // device status word of the workspace, cleared by the first CTA
+  int q_heads = 0, kv_heads = 0, seq_len = 0, head_dim = 0, span_begin = 0, span_len = 0;
+  int soft_lo = 0, soft_n = 0;  // keys the softmax runs over: [soft_lo, soft_lo + soft_n)
+  float scale = 0.f;
+  // Tail run by the last CTA of a sequence to finish (all null/zero: no tail):
+  int* counters = nullptr;     // [batch], zero before the launch
+  float* scores = nullptr;     // [batch][span_len] head mean (optional)
+  int32_t* kept = nullptr;     // [batch][k_keep] top-k of the head mean, ascending (optional)
+  int k_keep = 0;
 };
 
 // One CTA per (query head, sequence).  Dynamic shared memory: q[head_dim] floats | z[soft_n] floats.
-// Eight lanes share one key row (each lane 16-byte pieces, fp32 accumulate, 3 shuffles).
-template <typename T>
+// Eight lanes share one key row (16-byte pieces, fp32 accumulate, 3 shuffles); each 8-lane group has
+// four rows in flight.  VPS = 16-byte pieces per lane and row when that is a compile-time constant
+// (head_dim / (8 lanes * elements per piece)), 0 for any other head_dim.
+// With `counters` set, the CTA that finishes a sequence last sums the per-head probabilities in head
+// order (the same fixed order whichever CTA it is), writes the head mean and/or its exact top-k.
+template <typename T, int VPS>
 __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   extern __shared__ __align__(16) float smem_f[];
   float* qs = smem_f;
   float* z = smem_f + p.head_dim;
   __shared__ float red[33];
+  __shared__ SelectScratch sc;
+  __shared__ int is_last;
   constexpr int E = Vec16<T>::kElems;
+  constexpr int R = 4;   // key rows in flight per 8-lane group
   const int h = blockIdx.x, b = blockIdx.y;
   if (h == 0 && b == 0 && threadIdx.x == 0 && p.status) *p.status = 0u;
   const int g = static_cast<int>((static_cast<long long>(h) * p.kv_heads) / p.q_heads);
@@ -37,25 +50,56 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   const int sub = threadIdx.x & 7;           // lane within the 8-lane group
   const int grp = threadIdx.x >> 3, ngrp = blockDim.x >> 3;
   float local_max = -INFINITY;
-  for (int j0 = 0; j0 < p.soft_n; j0 += ngrp) {   // uniform trip count: shuffles stay converged
-    const int j = j0 + grp;
-    float acc = 0.f;
-    if (j < p.soft_n) {
-      const uint4* row = reinterpret_cast<const uint4*>(kb + static_cast<size_t>(j) * p.head_dim);
-      for (int v = sub; v < vecs; v += 8) {
-        float kv[E];
-        Vec16<T>::unpack(ld_nc_16(row + v), kv);
+  for (int j0 = 0; j0 < p.soft_n; j0 += R * ngrp) {   // uniform trip count: shuffles stay converged
+    float acc[R];
+    if constexpr (VPS > 0) {
+      uint4 raw[R][VPS];
 #pragma unroll
-        for (int e = 0; e < E; ++e) acc = fmaf(kv[e], qs[v * E + e], acc);
+      for (int u = 0; u < R; ++u) {
+        const int j = j0 + u * ngrp + grp;
+        const uint4* row = reinterpret_cast<const uint4*>(kb + static_cast<size_t>(min(j, p.soft_n - 1)) * p.head_dim);
+#pragma unroll
+        for (int i = 0; i < VPS; ++i) raw[u][i] = ld_nc_16(row + sub + 8 * i);
+      }
+#pragma unroll
+      for (int u = 0; u < R; ++u) {
+        acc[u] = 0.f;
+#pragma unroll
+        for (int i = 0; i < VPS; ++i) {
+          float kv[E];
+          Vec16<T>::unpack(raw[u][i], kv);
+#pragma unroll
+          for (int e = 0; e < E; ++e) acc[u] = fmaf(kv[e], qs[(sub + 8 * i) * E + e], acc[u]);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < R; ++u) {
+        const int j = j0 + u * ngrp + grp;
+        acc[u] = 0.f;
+        if (j < p.soft_n) {
+          const uint4* row = reinterpret_cast<const uint4*>(kb + static_cast<size_t>(j) * p.head_dim);
+          for (int v = sub; v < vecs; v += 8) {
+            float kv[E];
+            Vec16<T>::unpack(ld_nc_16(row + v), kv);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[u] = fmaf(kv[e], qs[v * E + e], acc[u]);
+          }
+        }
       }
     }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-    if (j < p.soft_n) {
-      acc *= p.scale;
-      if (sub == 0) z[j] = acc;
-      local_max = fmaxf(local_max, acc);
+#pragma unroll
+    for (int u = 0; u < R; ++u) {
+      const int j = j0 + u * ngrp + grp;
+      float a = acc[u];
+      a += __shfl_xor_sync(0xffffffffu, a, 1);
+      a += __shfl_xor_sync(0xffffffffu, a, 2);
+      a += __shfl_xor_sync(0xffffffffu, a, 4);
+      if (j < p.soft_n) {
+        a *= p.scale;
+        if (sub == 0) z[j] = a;
+        local_max = fmaxf(local_max, a);
+      }
     }
   }
   // block max
@@ -90,16 +134,42 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   float* out = p.probs + (static_cast<size_t>(b) * p.q_heads + h) * p.span_len;
   const int off = p.span_begin - p.soft_lo;
   for (int j = threadIdx.x; j < p.span_len; j += blockDim.x) out[j] = z[off + j] * inv;
+
+  if (!p.counters) return;
+  // ---- tail: whoever finishes this sequence last reduces over the heads
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) is_last = (atomicAdd(&p.counters[b], 1) == p.q_heads - 1);
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  uint32_t* keys = reinterpret_cast<uint32_t*>(z);   // span_len <= soft_n entries fit
+  const float* base = p.probs + static_cast<size_t>(b) * p.q_heads * p.span_len;
+  for (int j = threadIdx.x; j < p.span_len; j += blockDim.x) {
+    float acc = 0.f;
+    int hh = 0;
+    for (; hh + 8 <= p.q_heads; hh += 8) {
+      float a[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) a[u] = __ldcg(base + static_cast<size_t>(hh + u) * p.span_len + j);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) acc += a[u];
+    }
+    for (; hh < p.q_heads; ++hh) acc += __ldcg(base + static_cast<size_t>(hh) * p.span_len + j);
+    acc /= static_cast<float>(p.q_heads);
+    if (p.scores) p.scores[static_cast<size_t>(b) * p.span_len + j] = acc;
+    keys[j] = float_to_key(acc);
+  }
+  __syncthreads();
+  if (p.kept && p.k_keep > 0)
+    block_topk_emit(keys, p.span_len, p.k_keep, sc, p.kept + static_cast<size_t>(b) * p.k_keep);
 }
 
 inline size_t qk_smem_bytes(int head_dim, int soft_n) {
   return (static_cast<size_t>(head_dim) + soft_n) * sizeof(float) + 16;
 }
 
-// Host-side launch shared by both entry points.
+// Host-side launch shared by the entry points.
 vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStream_t stream);
-
-// scores[b][j] = (1/q_heads) * sum_h probs[b][h][j], h ascending.
-__global__ void head_mean_kernel(const float* probs, float* scores, int q_heads, int span_len);
 
 }  // namespace vscan

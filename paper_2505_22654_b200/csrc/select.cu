@@ -1,5 +1,7 @@
 // vscan_select_global_local: local scan (Eq. 3), global scan (Eq. 2) over the complement, union.
 // One CTA per encoder instance; all state of the instance lives in shared memory.
+#include <type_traits>
+
 #include "topk.cuh"
 
 namespace vscan {
@@ -7,12 +9,36 @@ namespace vscan {
 struct SelectParams {
   const float* scores_global;
   const float* scores_local;
+  // fused form: the scores are the head means of these attention rows (Eq. 2), taken here
+  const void* attn_global;
+  const void* attn_local;
+  float* scores_global_out;   // optional
+  float* scores_local_out;    // optional
+  int heads, row_len, cls_offset;
   int32_t* kept_idx;
   uint8_t* kept_mask;
   int n, frames, grid_h, grid_w, win_h, win_w, k_w, k_g, windows, wins_per_row, wins_per_frame;
 };
 
+// Head mean of one token's attention entries, heads ascending (same arithmetic as the ROW-mode score).
+template <typename T>
+__device__ __forceinline__ float head_mean_of(const T* base, int heads, int row_len) {
+  float acc = 0.f;
+  int h = 0;
+  for (; h + 8 <= heads; h += 8) {
+    float a[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) a[u] = to_float(base[static_cast<size_t>(h + u) * row_len]);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += a[u];
+  }
+  for (; h < heads; ++h) acc += to_float(base[static_cast<size_t>(h) * row_len]);
+  return acc / static_cast<float>(heads);
+}
+
 // dynamic shared memory: keys_g[n] | keys_l[n] | taken[n] (bytes)
+// T = void: scores are read; T = element type: scores are computed from the attention rows.
+template <typename T>
 __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* keys_g = reinterpret_cast<uint32_t*>(smem_raw);
@@ -21,12 +47,27 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
   __shared__ SelectScratch sc;
 
   const int b = blockIdx.x;
-  const float* sg = p.scores_global + static_cast<size_t>(b) * p.n;
-  const float* sl = p.scores_local + static_cast<size_t>(b) * p.n;
-  for (int i = threadIdx.x; i < p.n; i += blockDim.x) {
-    keys_g[i] = float_to_key(sg[i]);
-    keys_l[i] = float_to_key(sl[i]);
-    taken[i] = 0;
+  if constexpr (std::is_void<T>::value) {
+    const float* sg = p.scores_global + static_cast<size_t>(b) * p.n;
+    const float* sl = p.scores_local + static_cast<size_t>(b) * p.n;
+    for (int i = threadIdx.x; i < p.n; i += blockDim.x) {
+      keys_g[i] = float_to_key(sg[i]);
+      keys_l[i] = float_to_key(sl[i]);
+      taken[i] = 0;
+    }
+  } else {
+    const size_t inst = static_cast<size_t>(b) * p.heads * p.row_len + p.cls_offset;
+    const T* ag = static_cast<const T*>(p.attn_global) + inst;
+    const T* al = static_cast<const T*>(p.attn_local) + inst;
+    for (int i = threadIdx.x; i < p.n; i += blockDim.x) {
+      const float g = head_mean_of(ag + i, p.heads, p.row_len);
+      const float l = p.attn_local == p.attn_global ? g : head_mean_of(al + i, p.heads, p.row_len);
+      if (p.scores_global_out) p.scores_global_out[static_cast<size_t>(b) * p.n + i] = g;
+      if (p.scores_local_out) p.scores_local_out[static_cast<size_t>(b) * p.n + i] = l;
+      keys_g[i] = float_to_key(g);
+      keys_l[i] = float_to_key(l);
+      taken[i] = 0;
+    }
   }
   __syncthreads();
 
@@ -39,8 +80,9 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
                 wc = w % p.wins_per_row;
       const int base = f * p.grid_h * p.grid_w + wr * p.win_h * p.grid_w + wc * p.win_w;
       const int win_w = p.win_w, grid_w = p.grid_w;
-      warp_select_mark(keys_l, m, p.k_w,
-                       [=](int q) { return base + (q / win_w) * grid_w + (q % win_w); }, taken);
+      auto token_of = [=](int q) { return base + (q / win_w) * grid_w + (q % win_w); };
+      if (m <= 64) warp_rank_mark(keys_l, m, p.k_w, token_of, taken);
+      else warp_select_mark(keys_l, m, p.k_w, token_of, taken);
     }
   }
   __syncthreads();
@@ -92,43 +134,102 @@ using namespace vscan;
 
 extern "C" size_t vscan_select_workspace_bytes(const vscan_select_desc*) { return 0; }
 
-extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
-                                                  size_t /*workspace_bytes*/, void* stream) {
-  if (d && d->instances == 0) return VSCAN_OK;  // empty batch
-  if (!d || !d->scores_global || !d->scores_local || !d->kept_idx) return VSCAN_ERR_INVALID_ARG;
-  if (d->instances < 0 || d->frames <= 0 || d->grid_h <= 0 || d->grid_w <= 0 || d->win_h <= 0 ||
-      d->win_w <= 0)
+static vscan_status validate_grid(const vscan_select_desc* d, long long* n_out, int* windows_out, long long* k1_out) {
+  if (d->instances < 0 || d->frames <= 0 || d->grid_h <= 0 || d->grid_w <= 0 || d->win_h <= 0 || d->win_w <= 0)
     return VSCAN_ERR_INVALID_ARG;
   if (d->grid_h % d->win_h || d->grid_w % d->win_w) return VSCAN_ERR_INVALID_ARG;
   const long long n = 1ll * d->frames * d->grid_h * d->grid_w;
   if (n > 16384) return VSCAN_ERR_UNSUPPORTED;
+  if (d->instances > 65535) return VSCAN_ERR_UNSUPPORTED;
   const int windows = d->frames * (d->grid_h / d->win_h) * (d->grid_w / d->win_w);
   if (d->k_per_window < 0 || d->k_per_window > d->win_h * d->win_w) return VSCAN_ERR_INVALID_ARG;
   const long long local_total = 1ll * windows * d->k_per_window;
   if (d->k_global < 0 || d->k_global > n - local_total) return VSCAN_ERR_INVALID_ARG;
-  const long long k1 = local_total + d->k_global;
-  if (!aligned16(d->scores_global) || !aligned16(d->scores_local) || !aligned16(d->kept_idx))
-    return VSCAN_ERR_INVALID_ARG;
-  const size_t sbytes = static_cast<size_t>(d->instances) * n * 4, obytes = static_cast<size_t>(d->instances) * k1 * 4;
-  if (overlaps(d->kept_idx, obytes, d->scores_global, sbytes) ||
-      overlaps(d->kept_idx, obytes, d->scores_local, sbytes) ||
-      overlaps(d->kept_mask, static_cast<size_t>(d->instances) * n, d->scores_global, sbytes) ||
-      overlaps(d->kept_mask, static_cast<size_t>(d->instances) * n, d->scores_local, sbytes) ||
-      overlaps(d->kept_mask, static_cast<size_t>(d->instances) * n, d->kept_idx, obytes))
-    return VSCAN_ERR_INVALID_ARG;
-  if (d->instances == 0) return VSCAN_OK;
+  *n_out = n; *windows_out = windows; *k1_out = local_total + d->k_global;
+  return VSCAN_OK;
+}
 
-  SelectParams p;
+static void fill_params(SelectParams& p, const vscan_select_desc* d, long long n, int windows) {
+  p = SelectParams{};
   p.scores_global = d->scores_global; p.scores_local = d->scores_local;
   p.kept_idx = d->kept_idx; p.kept_mask = d->kept_mask;
   p.n = static_cast<int>(n); p.frames = d->frames; p.grid_h = d->grid_h; p.grid_w = d->grid_w;
   p.win_h = d->win_h; p.win_w = d->win_w; p.k_w = d->k_per_window; p.k_g = d->k_global;
   p.windows = windows; p.wins_per_row = d->grid_w / d->win_w;
   p.wins_per_frame = (d->grid_h / d->win_h) * p.wins_per_row;
+}
+
+// One warp per window while there are enough windows to fill the block.
+static int select_threads(long long n, int windows) { return n > 2048 ? 1024 : (windows > 8 ? 512 : 256); }
+
+extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
+                                                  size_t /*workspace_bytes*/, void* stream) {
+  if (d && d->instances == 0) return VSCAN_OK;  // empty batch
+  if (!d || !d->scores_global || !d->scores_local || !d->kept_idx) return VSCAN_ERR_INVALID_ARG;
+  long long n, k1;
+  int windows;
+  vscan_status vs = validate_grid(d, &n, &windows, &k1);
+  if (vs != VSCAN_OK) return vs;
+  if (!aligned16(d->scores_global) || !aligned16(d->scores_local) || !aligned16(d->kept_idx))
+    return VSCAN_ERR_INVALID_ARG;
+  const size_t sbytes = static_cast<size_t>(d->instances) * n * 4, obytes = static_cast<size_t>(d->instances) * k1 * 4;
+  const size_t mbytes = static_cast<size_t>(d->instances) * n;
+  if (overlaps(d->kept_idx, obytes, d->scores_global, sbytes) || overlaps(d->kept_idx, obytes, d->scores_local, sbytes) ||
+      overlaps(d->kept_mask, mbytes, d->scores_global, sbytes) || overlaps(d->kept_mask, mbytes, d->scores_local, sbytes) ||
+      overlaps(d->kept_mask, mbytes, d->kept_idx, obytes))
+    return VSCAN_ERR_INVALID_ARG;
+
+  SelectParams p;
+  fill_params(p, d, n, windows);
   const size_t smem = static_cast<size_t>(n) * 9 + 16;
-  VSCAN_CUDA_TRY(allow_smem(select_kernel, smem));
-  const int threads = n <= 2048 ? 256 : 1024;
+  VSCAN_CUDA_TRY(allow_smem(select_kernel<void>, smem));
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  VSCAN_LAUNCH("select", st, select_kernel<<<d->instances, threads, smem, st>>>(p));
+  VSCAN_LAUNCH("select", st, select_kernel<void><<<d->instances, select_threads(n, windows), smem, st>>>(p));
+  return VSCAN_OK;
+}
+
+extern "C" vscan_status vscan_score_select(const vscan_score_select_desc* d, void* stream) {
+  if (d && d->select.instances == 0) return VSCAN_OK;  // empty batch
+  if (!d || !d->attn_global || !d->attn_local || !d->select.kept_idx) return VSCAN_ERR_INVALID_ARG;
+  if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
+  const vscan_select_desc* sd = &d->select;
+  long long n, k1;
+  int windows;
+  vscan_status vs = validate_grid(sd, &n, &windows, &k1);
+  if (vs != VSCAN_OK) return vs;
+  if (d->heads <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + n) return VSCAN_ERR_INVALID_ARG;
+  const void* ptrs[] = {d->attn_global, d->attn_local, sd->kept_idx, sd->scores_global, sd->scores_local};
+  for (const void* ptr : ptrs)
+    if (ptr && !aligned16(ptr)) return VSCAN_ERR_INVALID_ARG;
+  const size_t abytes = static_cast<size_t>(sd->instances) * d->heads * d->row_len * dtype_bytes(d->dtype);
+  const size_t sbytes = static_cast<size_t>(sd->instances) * n * 4, obytes = static_cast<size_t>(sd->instances) * k1 * 4;
+  const size_t mbytes = static_cast<size_t>(sd->instances) * n;
+  struct Rng { const void* p; size_t n; };
+  const Rng outs[] = {{sd->kept_idx, obytes}, {sd->kept_mask, mbytes}, {sd->scores_global, sbytes}, {sd->scores_local, sbytes}};
+  for (const Rng& o : outs) {
+    if (overlaps(o.p, o.n, d->attn_global, abytes) || overlaps(o.p, o.n, d->attn_local, abytes)) return VSCAN_ERR_INVALID_ARG;
+    for (const Rng& o2 : outs)
+      if (o.p != o2.p && overlaps(o.p, o.n, o2.p, o2.n)) return VSCAN_ERR_INVALID_ARG;
+  }
+  if (sd->scores_global && sd->scores_global == sd->scores_local && d->attn_global != d->attn_local)
+    return VSCAN_ERR_INVALID_ARG;
+
+  SelectParams p;
+  fill_params(p, sd, n, windows);
+  p.scores_global = nullptr; p.scores_local = nullptr;
+  p.attn_global = d->attn_global; p.attn_local = d->attn_local;
+  p.scores_global_out = const_cast<float*>(sd->scores_global);
+  p.scores_local_out = const_cast<float*>(sd->scores_local);
+  p.heads = d->heads; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
+  const size_t smem = static_cast<size_t>(n) * 9 + 16;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int threads = select_threads(n, windows);
+  if (d->dtype == VSCAN_F32) {
+    VSCAN_CUDA_TRY(allow_smem(select_kernel<float>, smem));
+    VSCAN_LAUNCH("score_select", st, select_kernel<float><<<sd->instances, threads, smem, st>>>(p));
+  } else {
+    VSCAN_CUDA_TRY(allow_smem(select_kernel<__nv_bfloat16>, smem));
+    VSCAN_LAUNCH("score_select", st, select_kernel<__nv_bfloat16><<<sd->instances, threads, smem, st>>>(p));
+  }
   return VSCAN_OK;
 }

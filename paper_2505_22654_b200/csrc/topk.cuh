@@ -71,6 +71,31 @@ __device__ __forceinline__ void block_radix_select(const uint32_t* keys, const u
   need = k_rem;
 }
 
+// Block-wide: the k largest of keys[0..n) (equal keys to the lowest index) written in ascending index
+// order to out[0..k).  n <= 64 * blockDim.x.  All threads must call; 1 <= k <= n.
+__device__ __forceinline__ void block_topk_emit(const uint32_t* keys, int n, int k, SelectScratch& sc, int32_t* out) {
+  uint32_t thr;
+  int need;
+  block_radix_select(keys, nullptr, n, k, sc, thr, need);
+  const int per = (n + blockDim.x - 1) / blockDim.x;
+  const int lo = min(n, static_cast<int>(threadIdx.x) * per), hi = min(n, lo + per);
+  int eq_local = 0;
+  for (int i = lo; i < hi; ++i) eq_local += (keys[i] == thr);
+  int total;
+  int eq_before = block_exclusive_scan(eq_local, sc.warp_sums, total);
+  int kept_local = 0;
+  unsigned long long flags = 0;
+  for (int i = lo; i < hi; ++i) {
+    const uint32_t key = keys[i];
+    bool keep = key > thr;
+    if (key == thr) { keep = eq_before < need; ++eq_before; }
+    if (keep) { flags |= 1ull << (i - lo); ++kept_local; }
+  }
+  int pos = block_exclusive_scan(kept_local, sc.warp_sums, total);
+  for (int i = lo; i < hi; ++i)
+    if ((flags >> (i - lo)) & 1ull) { if (pos < k) out[pos] = i; ++pos; }
+}
+
 // Warp-wide bitwise select over m candidates enumerated by `token_of(p)`, p in [0, m), ascending
 // in p.  Marks the k winners in `selected` (shared memory, one byte per token).  0 <= k <= m.
 template <typename TokenOf>
@@ -111,6 +136,33 @@ __device__ __forceinline__ void warp_select_mark(const uint32_t* keys, int m, in
     if (gt || (eq && rank < k_rem)) selected[t] = 1;
     taken_eq += __popc(eq_mask);
   }
+}
+
+// Warp-wide exact top-k for small candidate sets (m <= 64) by rank counting: candidate p is kept
+// iff fewer than k candidates beat it (larger key, or equal key and smaller p).  Two candidates per
+// lane live in registers; the keys are passed around with shuffles, no shared-memory traffic.
+template <typename TokenOf>
+__device__ __forceinline__ void warp_rank_mark(const uint32_t* keys, int m, int k, TokenOf token_of,
+                                               uint8_t* selected) {
+  if (k <= 0) return;
+  const int lane = threadIdx.x & 31;
+  const int p0 = lane, p1 = lane + 32;
+  const int t0 = p0 < m ? token_of(p0) : 0, t1 = p1 < m ? token_of(p1) : 0;
+  const uint32_t k0 = p0 < m ? keys[t0] : 0u, k1 = p1 < m ? keys[t1] : 0u;
+  int r0 = 0, r1 = 0;
+  const int m0 = min(m, 32);
+  for (int j = 0; j < m0; ++j) {
+    const uint32_t kj = __shfl_sync(0xffffffffu, k0, j);
+    r0 += (kj > k0) || (kj == k0 && j < p0);
+    r1 += (kj >= k1);                       // every j < 32 precedes p1
+  }
+  for (int j = 32; j < m; ++j) {
+    const uint32_t kj = __shfl_sync(0xffffffffu, k1, j - 32);
+    r0 += (kj > k0);                        // every j >= 32 follows p0
+    r1 += (kj > k1) || (kj == k1 && j < p1);
+  }
+  if (p0 < m && r0 < k) selected[t0] = 1;
+  if (p1 < m && r1 < k) selected[t1] = 1;
 }
 
 }  // namespace vscan

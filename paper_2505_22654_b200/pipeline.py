@@ -14,7 +14,7 @@ from . import binding as vb
 class VScanReducer:
     def __init__(self, *, dtype, instances, frames, grid_h, grid_w, cls, D, H, win_h, win_w, k_w, k_g,
                  B, n_sys, n_vis, n_txt, Dh, Hq, Hkv, d, k2, pos_planes=1, scale=None,
-                 softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, device="cuda"):
+                 softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, fused_select=True, device="cuda"):
         self.dtype = torch.float32 if dtype in ("f32", torch.float32) else torch.bfloat16
         self.instances, self.frames, self.grid_h, self.grid_w, self.cls = instances, frames, grid_h, grid_w, cls
         self.D, self.H, self.win_h, self.win_w, self.k_w, self.k_g = D, H, win_h, win_w, k_w, k_g
@@ -27,7 +27,7 @@ class VScanReducer:
         self.S = n_sys + n_vis + n_txt
         self.S_out = self.S - n_vis + k2
         self.scale = float(scale if scale is not None else d ** -0.5)
-        self.softmax_span, self.merge_path = softmax_span, merge_path
+        self.softmax_span, self.merge_path, self.fused_select = softmax_span, merge_path, fused_select
         dev, dt = device, self.dtype
         self.scores_g = torch.empty((instances, self.N), dtype=torch.float32, device=dev)
         self.scores_l = torch.empty((instances, self.N), dtype=torch.float32, device=dev)
@@ -53,10 +53,15 @@ class VScanReducer:
 
     # ---- device-resident pass: the four library calls on the current stream
     def stage1(self, attn_g, attn_l, x):
-        vb.vscan_score_row(attn_g, self.cls, self.N, out=self.scores_g)
-        vb.vscan_score_row(attn_l, self.cls, self.N, out=self.scores_l)
-        vb.vscan_select_global_local(self.scores_g, self.scores_l, self.frames, self.grid_h, self.grid_w,
-                                     self.win_h, self.win_w, self.k_w, self.k_g, out=self.kept_idx)
+        if self.fused_select:      # Eq. 2 and Eq. 3 in one launch; the head means are still written out
+            vb.vscan_score_select(attn_g, attn_l, self.cls, self.frames, self.grid_h, self.grid_w, self.win_h,
+                                  self.win_w, self.k_w, self.k_g, out=self.kept_idx, scores_global=self.scores_g,
+                                  scores_local=self.scores_l)
+        else:
+            vb.vscan_score_row(attn_g, self.cls, self.N, out=self.scores_g)
+            vb.vscan_score_row(attn_l, self.cls, self.N, out=self.scores_l)
+            vb.vscan_select_global_local(self.scores_g, self.scores_l, self.frames, self.grid_h, self.grid_w,
+                                         self.win_h, self.win_w, self.k_w, self.k_g, out=self.kept_idx)
         if not self._sized:
             self._reserve(x)
         vb.vscan_merge(x, self.cls, self.kept_idx, n_tokens=self.N, path=self.merge_path, out=self.merged,

@@ -79,6 +79,31 @@ def test_select_uniform_scores_take_first_indices_and_aliasing():
     assert {0, 1, 6, 7, 144, 145}.issubset(set(got[0].tolist()))
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 24, 24, 6, 6, 2, 32, 1, 16), (2, 6, 8, 3, 4, 5, 20, 0, 5),
+                                   (1, 16, 16, 16, 16, 40, 9, 1, 3), (16, 32, 32, 8, 8, 4, 1024, 0, 16)])
+def test_score_select_fused_matches_oracle(dtype, shape):
+    F, Gh, Gw, wh, ww, k_w, k_g, c, H = shape
+    N, B = F * Gh * Gw, 2
+    cfg = small_cfg(dtype, frames=F, grid_h=Gh, grid_w=Gw, win_h=wh, win_w=ww, k_w=k_w, k_g=k_g, cls=c, H=H, C=1, B=B)
+    ag = round_to_dtype(RNG.random((B, H, N + c)).astype(np.float32) / N, dtype)
+    al = round_to_dtype(RNG.random((B, H, N + c)).astype(np.float32) / N, dtype)
+    plant.plant_stage1_scores(cfg, ag, al)
+    sg = torch.empty((B, N), dtype=torch.float32, device="cuda"); sl = torch.empty_like(sg)
+    kept = vs.vscan_score_select(dev(ag, dtype), dev(al, dtype), c, F, Gh, Gw, wh, ww, k_w, k_g,
+                                 scores_global=sg, scores_local=sl).cpu().numpy()
+    for b in range(B):
+        rg, rl = vo.score_row(ag[b], c), vo.score_row(al[b], c)
+        assert np.abs(sg[b].cpu().numpy() - rg).max() <= TOL_SCORE and np.abs(sl[b].cpu().numpy() - rl).max() <= TOL_SCORE
+        np.testing.assert_array_equal(kept[b], vo.select_global_local(rg, rl, F, Gh, Gw, wh, ww, k_w, k_g)[0])
+    # same buffer for both scans, no score outputs: the decisions are taken on the kernel's own fp32
+    # head means (returned above), so the oracle fed with exactly those values must agree bit for bit
+    kept2 = vs.vscan_score_select(dev(ag, dtype), dev(ag, dtype), c, F, Gh, Gw, wh, ww, k_w, k_g).cpu().numpy()
+    for b in range(B):
+        g32 = sg[b].cpu().numpy()
+        np.testing.assert_array_equal(kept2[b], vo.select_global_local(g32, g32, F, Gh, Gw, wh, ww, k_w, k_g)[0])
+
+
 # ------------------------------------------------------------------ vscan_merge
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("path", ["simt", "auto"])
