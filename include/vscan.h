@@ -58,7 +58,10 @@ typedef enum { VSCAN_SPAN_ONLY = 0, VSCAN_SPAN_FULL = 1 } vscan_softmax_span;
 typedef enum {
   VSCAN_MERGE_AUTO = 0,   /* tensor cores for bf16 when the shape allows, else CUDA cores */
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
-  VSCAN_MERGE_TENSOR = 2  /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory */
+  VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group means in a
+                             second kernel */
+  VSCAN_MERGE_FUSED = 3   /* norms, tcgen05 similarity + arg-max and group means in one kernel, one cluster of
+                             CTAs per instance (bf16, n_kept <= 256, n_tokens <= 8192) */
 } vscan_merge_path;
 
 /* ---------------------------------------------------------------------------------------------

@@ -259,7 +259,8 @@ using namespace vscan;
 static vscan_status validate_merge(const vscan_merge_desc* d) {
   if (!d || !d->x || !d->kept_idx || !d->merged) return VSCAN_ERR_INVALID_ARG;
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
-  if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR)
+  if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR &&
+      d->path != VSCAN_MERGE_FUSED)
     return VSCAN_ERR_INVALID_ARG;
   if (d->instances < 0 || d->n_tokens <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + d->n_tokens ||
       d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
@@ -318,6 +319,19 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   p.merged = d->merged; p.counts = d->counts;
   p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
+
+  // fused kernel: one launch for the whole call
+  if (d->path == VSCAN_MERGE_FUSED) {   // measured slower than the two-kernel tensor path: opt-in only
+    if (merge_fused_supported(d->dtype, p)) {
+      p.assign = d->assign;   // optional output only; the fused kernel keeps assignments on chip
+      VSCAN_CUDA_TRY(cudaMemsetAsync(p.status, 0, sizeof(uint32_t), stream));
+      st = launch_merge_fused(p, stream);
+      if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_FUSED) return st;
+      p.assign = d->assign ? d->assign : ws_assign;
+    } else if (d->path == VSCAN_MERGE_FUSED) {
+      return VSCAN_ERR_UNSUPPORTED;
+    }
+  }
 
   bool tensor = false;
   if (d->path == VSCAN_MERGE_TENSOR) {

@@ -23,5 +23,9 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 // cannot take.
 vscan_status launch_assign_tensor(const MergeParams& p, cudaStream_t stream);
 bool assign_tensor_supported(int dtype, const MergeParams& p);
+// Norms, assignment and group means in one kernel (bf16, at most 256 kept tokens and 8192 tokens per
+// instance).  Writes merged / assign / counts directly; needs no inv_norm or assign scratch.
+vscan_status launch_merge_fused(const MergeParams& p, cudaStream_t stream);
+bool merge_fused_supported(int dtype, const MergeParams& p);
 
 }  // namespace vscan

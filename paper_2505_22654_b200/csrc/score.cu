@@ -28,10 +28,13 @@ static vscan_status launch_qk_typed(const QkParams& p, int batch, size_t smem, c
   constexpr int E = Vec16<T>::kElems;
   dim3 grid(p.q_heads, batch);
   const int vecs = p.head_dim / E;
+  // small CTAs keep every (head, sequence) pair of a typical batch resident at once; the top-k tail
+  // needs at most 64 keys per thread
+  const int threads = p.span_len <= 8192 ? 128 : 256;
 #define VSCAN_QK_CASE(VPS)                                                                          \
   do {                                                                                              \
     VSCAN_CUDA_TRY(allow_smem(qk_softmax_kernel<T, VPS>, smem));                                    \
-    VSCAN_LAUNCH("qk_softmax", stream, (qk_softmax_kernel<T, VPS><<<grid, 256, smem, stream>>>(p))); \
+    VSCAN_LAUNCH("qk_softmax", stream, (qk_softmax_kernel<T, VPS><<<grid, threads, smem, stream>>>(p))); \
     return VSCAN_OK;                                                                                \
   } while (0)
   if (vecs == 16) VSCAN_QK_CASE(2);

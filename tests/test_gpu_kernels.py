@@ -166,7 +166,8 @@ def test_merge_exact_ties_and_duplicates():
 
 @pytest.mark.parametrize("N,D,K1,c", [(576, 1024, 64, 1), (576, 1024, 192, 1), (300, 72, 17, 0), (130, 264, 130, 1),
                                       (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0)])
-def test_merge_tensor_path_matches_oracle(N, D, K1, c):
+@pytest.mark.parametrize("path", ["tensor", "fused"])
+def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     """The tcgen05 path on its own (path = TENSOR): tile tails, kept counts that are not multiples of
     16, more than 256 kept tokens (several accumulator rounds), feature dims that are not multiples
     of 64."""
@@ -174,9 +175,15 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c):
     x = round_to_dtype(RNG.standard_normal((2, N + c, D)).astype(np.float32), "bf16")
     kept = np.stack([np.sort(RNG.choice(N, K1, replace=False)) for _ in range(2)])
     plant.plant_merge(cfg, x, kept)
+    if path == "fused" and K1 > 256:
+        with pytest.raises(vs.VScanError) as e:
+            vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_FUSED)
+        assert e.value.status == 2       # more kept tokens than one accumulator holds: not this path
+        return
     ws = vs.Workspace(1 << 20)
     merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
-                                            want_counts=True, path=vs.MERGE_TENSOR, workspace=ws)
+                                            want_counts=True, workspace=ws,
+                                            path=vs.MERGE_TENSOR if path == "tensor" else vs.MERGE_FUSED)
     assert vs.vscan_check(ws) == 0
     for b in range(2):
         m, a, cn = vo.merge(x[b], c, kept[b])
