@@ -46,6 +46,7 @@ def algorithmic_bytes(cfg) -> dict:
         "prune_topk": B * cfg.k2 * 4,
         "compact": B * 2 * cfg.S_out * (cfg.Dh * e + 2 * cfg.Hkv * cfg.d * e + cfg.pos_planes * 4),
     }
+    row["score_select"] = 2 * I * cfg.H * cfg.L * e + I * (2 * cfg.N * 4 + cfg.K1 * 4)   # fused Eq. 2 + Eq. 3
     row["step"] = 2 * row["row_mean"] + row["select"] + row["merge"] + row["qk_softmax"] + \
         row["prune_topk"] + row["compact"]
     return row

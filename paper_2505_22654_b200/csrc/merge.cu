@@ -143,14 +143,16 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 }
 
 // ------------------------------------------------------------------ group means
-// One CTA per (group of 8 slots, instance); warp w owns slot s0 + w.  The CTA first lists, in
-// ascending token order, the tokens assigned to its 8 slots; each warp then walks that list and
-// adds its members' rows in that order (fp32), two rows in flight.
+// One CTA per (group of 4 slots, instance); warp w owns slot s0 + w.  The CTA first lists, in
+// ascending token order, the tokens assigned to its slots; each warp then walks that list and adds
+// its members' rows in that order (fp32), R rows in flight.  Small CTAs keep a large group from
+// holding the resources of many finished warps.
 // dynamic shared memory: list[n_tokens] of (local slot << 24 | token)
-constexpr int kSlotsPerCta = 8;
+constexpr int kSlotsPerCta = 4;
+constexpr int kMeanThreads = kSlotsPerCta * 32;
 
-template <typename T, int VPL>
-__global__ void __launch_bounds__(256) group_mean_kernel(MergeParams p) {
+template <typename T, int VPL, int R>
+__global__ void __launch_bounds__(kMeanThreads) group_mean_kernel(MergeParams p) {
   constexpr int E = Vec16<T>::kElems;
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
@@ -190,30 +192,35 @@ __global__ void __launch_bounds__(256) group_mean_kernel(MergeParams p) {
       unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(w));
       count += __popc(mask);
       while (mask) {
-        const int l0 = __ffs(mask) - 1;
-        mask &= mask - 1;
-        const int l1 = mask ? __ffs(mask) - 1 : -1;
-        if (mask) mask &= mask - 1;
-        const int ta = static_cast<int>(__shfl_sync(0xffffffffu, entry, l0) & 0xFFFFFFu);
-        const int tb = l1 >= 0 ? static_cast<int>(__shfl_sync(0xffffffffu, entry, l1) & 0xFFFFFFu) : -1;
-        const uint4* ra = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(ta) * p.dim);
-        const uint4* rb = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tb < 0 ? ta : tb) * p.dim);
-        uint4 va[VPL], vb[VPL];
+        int tok[R];
 #pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-          const int v = v0 + lane + 32 * i;
-          if (v < vecs) { va[i] = ld_nc_16(ra + v); if (tb >= 0) vb[i] = ld_nc_16(rb + v); }
+        for (int r = 0; r < R; ++r) {
+          tok[r] = -1;
+          if (mask) {
+            const int l = __ffs(mask) - 1;
+            mask &= mask - 1;
+            tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
+          }
+        }
+        uint4 raw[R][VPL];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
+#pragma unroll
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
+          }
         }
 #pragma unroll
-        for (int i = 0; i < VPL; ++i) {
-          const int v = v0 + lane + 32 * i;
-          if (v < vecs) {
-            float f[E];
-            Vec16<T>::unpack(va[i], f);
+        for (int r = 0; r < R; ++r) {
+          if (tok[r] < 0) continue;
 #pragma unroll
-            for (int e = 0; e < E; ++e) acc[i][e] += f[e];
-            if (tb >= 0) {
-              Vec16<T>::unpack(vb[i], f);
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs) {
+              float f[E];
+              Vec16<T>::unpack(raw[r][i], f);
 #pragma unroll
               for (int e = 0; e < E; ++e) acc[i][e] += f[e];
             }
@@ -243,11 +250,11 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
   dim3 grid((p.n_kept + kSlotsPerCta - 1) / kSlotsPerCta, p.instances);
   if (p.dim / E <= 128) {
-    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4>, smem));
-    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 4><<<grid, 256, smem, stream>>>(p)));
+    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4, 4>, smem));
+    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 4, 4><<<grid, kMeanThreads, smem, stream>>>(p)));
   } else {
-    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8>, smem));
-    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 8><<<grid, 256, smem, stream>>>(p)));
+    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8, 2>, smem));
+    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 8, 2><<<grid, kMeanThreads, smem, stream>>>(p)));
   }
   return VSCAN_OK;
 }
@@ -341,19 +348,21 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
     tensor = assign_tensor_supported(d->dtype, p);
   }
 
-  dim3 ngrid((d->n_kept + 7) / 8, d->instances);
-  if (d->dtype == VSCAN_F32) VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p));
-  else VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p));
-
+  // the tensor path takes the norms of the kept rows itself; the CUDA-core path gets them from a
+  // small kernel of its own
+  st = VSCAN_ERR_UNSUPPORTED;
   if (tensor) {
+    VSCAN_CUDA_TRY(cudaMemsetAsync(p.status, 0, sizeof(uint32_t), stream));
     st = launch_assign_tensor(p, stream);
-    // a shape the tensor path cannot take (tensor-map limits) runs on the CUDA cores unless the
-    // caller insisted on tensor cores
-    if (st == VSCAN_ERR_UNSUPPORTED && d->path == VSCAN_MERGE_AUTO) st = launch_assign_simt(d->dtype, p, stream);
-  } else {
-    st = launch_assign_simt(d->dtype, p, stream);
+    if (st != VSCAN_OK && (st != VSCAN_ERR_UNSUPPORTED || d->path != VSCAN_MERGE_AUTO)) return st;
   }
-  if (st != VSCAN_OK) return st;
+  if (st == VSCAN_ERR_UNSUPPORTED) {   // CUDA cores (asked for, or a shape the tensor path cannot take)
+    dim3 ngrid((d->n_kept + 7) / 8, d->instances);
+    if (d->dtype == VSCAN_F32) VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<float><<<ngrid, 256, 0, stream>>>(p));
+    else VSCAN_LAUNCH("kept_inv_norm", stream, kept_inv_norm_kernel<__nv_bfloat16><<<ngrid, 256, 0, stream>>>(p));
+    st = launch_assign_simt(d->dtype, p, stream);
+    if (st != VSCAN_OK) return st;
+  }
 
   return d->dtype == VSCAN_F32 ? launch_group_mean<float>(p, stream)
                                : launch_group_mean<__nv_bfloat16>(p, stream);

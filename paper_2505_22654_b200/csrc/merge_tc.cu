@@ -4,7 +4,8 @@
 //   warp 0      TMA producer: the token tile (3-D tensor map over [instance][row][dim], 128B swizzle) and
 //               the kept rows, which are not contiguous, four rows per TMA gather
 //   warp 1      allocates tensor memory, issues the MMAs (one elected lane), commits to mbarriers
-//   warps 2-5   read the accumulator back (tcgen05.ld, one token row per thread), scale by 1/|m_s|
+//   warps 2-5   take the squared norms of the kept rows from the B stages while the MMAs run, then
+//               read the accumulator back (tcgen05.ld, one token row per thread), scale by 1/|m_s|
 //               and keep the running arg-max (lowest slot on ties); with more than 256 kept tokens
 //               two accumulators alternate so this overlaps the next round of MMAs
 // The similarity matrix never leaves the SM.  Every mbarrier wait is bounded: on expiry the CTA
@@ -55,7 +56,9 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
   const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    // a stage is free again once the MMAs that read it have completed and the four epilogue warps
+    // have taken the squared norms of its kept-row slice
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 5); }
     for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 4); }
     sh.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -144,15 +147,41 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     const int row = quarter * 32 + lane;      // token row of this thread within the tile
     float best_val = -INFINITY;
     int best_idx = 0;
+    int it = 0;
     bool ok = true;
     // Once `ok` drops the loop keeps running with its work skipped, so that the four warps execute
     // the same sequence of named barriers and warp-wide instructions whatever happens.
     for (int nc = 0; nc < p.n_chunks; ++nc) {
       const int n0 = nc * p.n_pad, acc = nc & 1, use = nc >> 1;
-      // scales of this n-chunk; the buffer was last read two chunks ago, before that chunk's arrive
-      for (int j = ptid; j < p.n_pad; j += 128) {
-        const int s_idx = n0 + j;
-        sh.inv_norm[acc][j] = s_idx < m.n_kept ? m.inv_norm[static_cast<size_t>(b) * m.n_kept + s_idx] : 0.f;
+      // |m_s|^2 of the kept rows of this n-chunk, accumulated from the B stages as they pass through
+      // shared memory (thread ptid owns rows ptid and ptid + 128)
+      float ss[2] = {0.f, 0.f};
+      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+        const int s = it % p.stages, round = it / p.stages;
+        if (ok) ok = mbar_wait_warp(&sh.full[s], round & 1, abort_flag);
+        if (!ok) continue;
+        const unsigned char* bt = tiles + s * stage_bytes + p.a_stage_bytes;
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int r = ptid + 128 * u;
+          if (r < p.n_pad) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              float f[8];
+              Vec16<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4*>(bt + r * 128 + ((j ^ (r & 7)) << 4)), f);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) ss[u] = fmaf(f[e], f[e], ss[u]);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.empty[s]);
+      }
+      // the buffer was last read two chunks ago, before that chunk's arrive on tmem_empty
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int r = ptid + 128 * u;
+        if (r < p.n_pad) sh.inv_norm[acc][r] = (n0 + r < m.n_kept) ? 1.f / fmaxf(sqrtf(ss[u]), 1e-12f) : 0.f;
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);

@@ -148,12 +148,19 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   for (int j = threadIdx.x; j < p.span_len; j += blockDim.x) {
     float acc = 0.f;
     int hh = 0;
-    for (; hh + 8 <= p.q_heads; hh += 8) {
-      float a[8];
+    for (; hh + 16 <= p.q_heads; hh += 16) {   // sixteen loads in flight, added in head order
+      float a[16];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) a[u] = __ldcg(base + static_cast<size_t>(hh + u) * p.span_len + j);
+      for (int u = 0; u < 16; ++u) a[u] = __ldcg(base + static_cast<size_t>(hh + u) * p.span_len + j);
 #pragma unroll
-      for (int u = 0; u < 8; ++u) acc += a[u];
+      for (int u = 0; u < 16; ++u) acc += a[u];
+    }
+    for (; hh + 4 <= p.q_heads; hh += 4) {
+      float a[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) a[u] = __ldcg(base + static_cast<size_t>(hh + u) * p.span_len + j);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) acc += a[u];
     }
     for (; hh < p.q_heads; ++hh) acc += __ldcg(base + static_cast<size_t>(hh) * p.span_len + j);
     acc /= static_cast<float>(p.q_heads);

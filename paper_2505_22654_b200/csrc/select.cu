@@ -25,12 +25,19 @@ template <typename T>
 __device__ __forceinline__ float head_mean_of(const T* base, int heads, int row_len) {
   float acc = 0.f;
   int h = 0;
-  for (; h + 8 <= heads; h += 8) {
-    float a[8];
+  for (; h + 16 <= heads; h += 16) {   // sixteen independent loads in flight, added in head order
+    T a[16];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) a[u] = to_float(base[static_cast<size_t>(h + u) * row_len]);
+    for (int u = 0; u < 16; ++u) a[u] = base[static_cast<size_t>(h + u) * row_len];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) acc += a[u];
+    for (int u = 0; u < 16; ++u) acc += to_float(a[u]);
+  }
+  for (; h + 4 <= heads; h += 4) {
+    T a[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) a[u] = base[static_cast<size_t>(h + u) * row_len];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc += to_float(a[u]);
   }
   for (; h < heads; ++h) acc += to_float(base[static_cast<size_t>(h) * row_len]);
   return acc / static_cast<float>(heads);
@@ -60,8 +67,9 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
     const T* ag = static_cast<const T*>(p.attn_global) + inst;
     const T* al = static_cast<const T*>(p.attn_local) + inst;
     for (int i = threadIdx.x; i < p.n; i += blockDim.x) {
+      const bool same = p.attn_local == p.attn_global;
       const float g = head_mean_of(ag + i, p.heads, p.row_len);
-      const float l = p.attn_local == p.attn_global ? g : head_mean_of(al + i, p.heads, p.row_len);
+      const float l = same ? g : head_mean_of(al + i, p.heads, p.row_len);
       if (p.scores_global_out) p.scores_global_out[static_cast<size_t>(b) * p.n + i] = g;
       if (p.scores_local_out) p.scores_local_out[static_cast<size_t>(b) * p.n + i] = l;
       keys_g[i] = float_to_key(g);
@@ -160,7 +168,7 @@ static void fill_params(SelectParams& p, const vscan_select_desc* d, long long n
 }
 
 // One warp per window while there are enough windows to fill the block.
-static int select_threads(long long n, int windows) { return n > 2048 ? 1024 : (windows > 8 ? 512 : 256); }
+static int select_threads(long long n, int windows) { return n > 2048 ? 1024 : (windows > 8 || n > 256 ? 512 : 256); }
 
 extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
                                                   size_t /*workspace_bytes*/, void* stream) {
