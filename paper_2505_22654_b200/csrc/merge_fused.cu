@@ -406,9 +406,9 @@ vscan_status launch_merge_fused(const MergeParams& m, cudaStream_t stream) {
   const cuuint32_t box_tail[3] = {tc::kChunkK, static_cast<cuuint32_t>(p.tail_rows), 1};
   void* base = const_cast<void*>(m.metric);
   if (encode(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS ||
       encode(&map_tail, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box_tail, elem,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return VSCAN_ERR_UNSUPPORTED;
   const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(m.metric_dim),
@@ -416,7 +416,7 @@ vscan_status launch_merge_fused(const MergeParams& m, cudaStream_t stream) {
   const cuuint64_t strides_b[1] = {static_cast<cuuint64_t>(m.metric_dim) * 2};
   const cuuint32_t box_b[2] = {tc::kChunkK, 1};
   if (encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims_b, strides_b, box_b, elem, CU_TENSOR_MAP_INTERLEAVE_NONE,
-             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return VSCAN_ERR_UNSUPPORTED;
 
   const size_t smem = static_cast<size_t>(p.tiles_bytes) + 1024 + (static_cast<size_t>(m.n_tokens) * 2 + 15) / 16 * 16;

@@ -281,7 +281,7 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   const cuuint32_t elem[3] = {1, 1, 1};
   CUresult r = encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(m.metric), dims, strides, box,
                       elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                      CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
   // kept rows: the same memory as a 2-D [all rows][dim] tensor, fetched four rows at a time
   CUtensorMap map_b;
@@ -290,7 +290,7 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   const cuuint64_t strides_b[1] = {static_cast<cuuint64_t>(m.metric_dim) * 2};
   const cuuint32_t box_b[2] = {tc::kChunkK, 1};
   r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(m.metric), dims_b, strides_b, box_b, elem,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
   const size_t smem = static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) + 1024;

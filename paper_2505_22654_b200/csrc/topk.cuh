@@ -29,19 +29,23 @@ __device__ __forceinline__ void block_radix_select(const uint32_t* keys, const u
     for (int i = threadIdx.x; i < 256; i += blockDim.x) sc.hist[i] = 0;
     __syncthreads();
     // Scores of one instance share their exponent, so in the first pass nearly every key falls into
-    // the same bin: lanes with equal digits are counted with one shared-memory atomic per warp.
-    for (int base = 0; base < n; base += blockDim.x) {
-      const int i = base + threadIdx.x;
-      bool valid = i < n && !(excluded && excluded[i]);
-      uint32_t digit = 0;
-      if (valid) {
-        const uint32_t key = keys[i];
-        valid = (key & mask) == prefix;
-        digit = (key >> shift) & 255u;
+    // the same bin: there lanes with equal digits are counted with one shared-memory atomic per warp.
+    // Later passes see spread-out digits and add directly.
+    if (shift == 24) {
+      for (int base = 0; base < n; base += blockDim.x) {
+        const int i = base + threadIdx.x;
+        const bool valid = i < n && !(excluded && excluded[i]);
+        const uint32_t digit = valid ? (keys[i] >> 24) : 0u;
+        const unsigned lane = threadIdx.x & 31;
+        const unsigned peers = __match_any_sync(0xffffffffu, valid ? digit : (256u + lane));
+        if (valid && lane == static_cast<unsigned>(__ffs(peers) - 1)) atomicAdd(&sc.hist[digit], __popc(peers));
       }
-      const unsigned lane = threadIdx.x & 31;
-      const unsigned peers = __match_any_sync(0xffffffffu, valid ? digit : (256u + lane));
-      if (valid && lane == static_cast<unsigned>(__ffs(peers) - 1)) atomicAdd(&sc.hist[digit], __popc(peers));
+    } else {
+      for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        if (excluded && excluded[i]) continue;
+        const uint32_t key = keys[i];
+        if ((key & mask) == prefix) atomicAdd(&sc.hist[(key >> shift) & 255u], 1);
+      }
     }
     __syncthreads();
     if (threadIdx.x < 32) {
