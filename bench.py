@@ -219,36 +219,35 @@ def build_sets(cfg, n_sets: int, device):
     gen_b = min(cfg.B, 32)
     s1, s2 = stage1_inputs(cfg, 0, gen_b * cfg.C), stage2_inputs(cfg, 0, gen_b)
 
-    def tile(a, total, axis=0):
-        reps = -(-total // a.shape[axis])
-        return np.concatenate([a] * reps, axis=axis).take(range(total), axis=axis) if reps > 1 else a
+    def tile(t, total, axis=0):
+        reps = -(-total // t.shape[axis])
+        if reps > 1:
+            t = torch.cat([t] * reps, dim=axis)
+        return t.narrow(axis, 0, total)
 
-    host = {"attn_g": tile(s1["attn_g"], cfg.instances), "attn_l": tile(s1["attn_l"], cfg.instances),
-            "x": tile(s1["x"], cfg.instances), "q_last": tile(s2["q_last"], cfg.B), "k": tile(s2["k"], cfg.B),
-            "v": tile(s2["v"], cfg.B), "hidden": tile(s2["hidden"], cfg.B)}
+    base = {name: torch.from_numpy(a).to(device=device, dtype=dt)
+            for name, a in (("attn_g", s1["attn_g"]), ("attn_l", s1["attn_l"]), ("x", s1["x"]),
+                            ("q_last", s2["q_last"]), ("k", s2["k"]), ("v", s2["v"]), ("hidden", s2["hidden"]))}
+    pos = torch.from_numpy(s2["pos_ids"]).to(device)
     sets = []
     for r in range(n_sets):
         d = {}
-        for name, a in host.items():
-            shift = r * (cfg.C if name in ("attn_g", "attn_l", "x") else 1)
-            d[name] = torch.from_numpy(np.roll(a, shift, axis=0)).to(device=device, dtype=dt).contiguous()
-        d["pos_ids"] = torch.from_numpy(tile(s2["pos_ids"], cfg.B, axis=1)).to(device).contiguous()
+        for name, t in base.items():
+            per_image = cfg.C if name in ("attn_g", "attn_l", "x") else 1
+            d[name] = tile(torch.roll(t, r * per_image, dims=0), cfg.B * per_image).contiguous()
+        d["pos_ids"] = tile(pos, cfg.B, axis=1).contiguous()
         sets.append(d)
     return sets
 
 
-def run_vscan(args, cfg):
+def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=True):
+    """Times one workload on this rank's GPU; rank 0 gets the JSON-able result dict, others None."""
     import torch
 
     import paper_2505_22654_b200 as vs
     from paper_2505_22654_b200 import binding as vb
 
-    rank, world, local_rank, dist = dist_setup(args.gpus)
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the VScan path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    vb.lib()
 
     n_sets = args.sets
     warmup = max(args.warmup, 3)
@@ -311,25 +310,28 @@ def run_vscan(args, cfg):
             per_kernel.setdefault(name, []).append(ms)
 
         # ---- end to end: pinned host buffers in and out, copies inside the timed region
+        e2e = None
         red, dev_in = reducers[0], sets[0]
-        host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in dev_in.items()}
-        outs = {"merged": red.merged, **{k: red.out2[k] for k in ("kept_vis", "hidden", "k", "v", "pos")}}
-        host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
-        e_steps = max(1, min(args.steps, 5))
-        red.run_host(host_in, host_out, dev_in)
-        stream.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(e_steps):
+        if with_e2e:
+            host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in dev_in.items()}
+            outs = {"merged": red.merged, **{k: red.out2[k] for k in ("kept_vis", "hidden", "k", "v", "pos")}}
+            host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
+            e_steps = max(1, min(args.steps, 5))
             red.run_host(host_in, host_out, dev_in)
-        e1.record(stream)
-        e1.synchronize()
-        e_ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
-        e2e = {"value": world * cfg.B * e_steps / (e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in.values())),
-               "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out.values())),
-               "steps": e_steps, "ms_per_step": e_ms / e_steps}
+            stream.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(e_steps):
+                red.run_host(host_in, host_out, dev_in)
+            e1.record(stream)
+            e1.synchronize()
+            e_ms = max_over_ranks(e0.elapsed_time(e1), dist, device)
+            e2e = {"value": world * cfg.B * e_steps / (e_ms * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in.values())),
+                   "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out.values())),
+                   "steps": e_steps, "ms_per_step": e_ms / e_steps}
 
+    line = None
     if rank == 0:
         peak, peak_kind = measured_peaks()
         alg = algorithmic_bytes(cfg)
@@ -350,7 +352,7 @@ def run_vscan(args, cfg):
             traffic = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json"))).get(dominant)
         except Exception:
             pass
-        cpu = time_oracle(cfg) if (world == 1 and not args.no_cpu_baseline) else None
+        cpu = time_oracle(cfg) if (world == 1 and with_cpu and not args.no_cpu_baseline) else None
         step_gbs = alg["step"] / (ms_step * 1e-3) / 1e9
         line = {
             "metric": METRIC, "value": world * cfg.B * args.steps / (ms_total * 1e-3), "unit": UNIT,
@@ -370,15 +372,70 @@ def run_vscan(args, cfg):
                          "algorithmic_bytes_per_launch": dom_bytes},
             "kernels": kernels,
             "merge": {"flops_per_step": merge_flops(cfg),
-                      "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names)},
+                      "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names),
+                      "assign_kernel": next((n for n in ("assign_tensor", "assign_simt", "merge_fused") if n in kernels), None)},
             "gpu_launches": launches_per_step * args.steps,
             "clocks": clocks,
             "e2e": e2e,
             "cpu_baseline": cpu,
         }
-        print(json.dumps(line))
+    del sets, reducers, graphs
+    torch.cuda.empty_cache()
+    return line
+
+
+def run_vscan(args, cfg):
+    import torch
+
+    from paper_2505_22654_b200 import binding as vb
+
+    rank, world, local_rank, dist = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the VScan path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    vb.lib()
+    if args.sweep:
+        run_sweep(args, rank, world, local_rank, dist)
+    else:
+        line = measure(args, cfg, rank, world, local_rank, dist)
+        if rank == 0:
+            print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_sweep(args, rank, world, local_rank, dist):
+    """Every named workload plus the batch x retention sweep at the 2880-token shape; one JSON line per
+    point.  For each retention level the merge is also timed on the CUDA-core path at batch 32, which
+    places the crossover between the two similarity paths."""
+    from synth import SWEEP_BATCHES, SWEEP_BUDGETS
+    peak_tf = 1395.5
+    try:
+        peak_tf = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
+    except Exception:
+        pass
+    points = [("config%d" % i, CONFIGS[i], 0) for i in (0, 1, 2, 3)]
+    points += [("sweep b=%d %s" % (b, r), sweep_config(b, r), 0) for r in SWEEP_BUDGETS for b in SWEEP_BATCHES]
+    points += [("simt b=32 %s" % r, sweep_config(32, r), 1) for r in SWEEP_BUDGETS]
+    points += [("tensor b=32 %s" % r, sweep_config(32, r), 2) for r in SWEEP_BUDGETS]
+    for label, cfg, path in points:
+        args.merge_path = path
+        steps = args.steps
+        args.steps = max(10, min(steps, int(2e5 / max(cfg.B, 1)) // 10 * 10)) if cfg.B > 64 else steps
+        line = measure(args, cfg, rank, world, local_rank, dist, with_e2e=False, with_cpu=False)
+        args.steps = steps
+        if rank != 0:
+            continue
+        k = line["kernels"]
+        assign = line["merge"]["assign_kernel"]
+        out = {"point": label, "workload": cfg.name, "B": cfg.B, "K1": cfg.K1, "dtype": cfg.dtype,
+               "images_per_s": round(line["value"], 1), "ms_per_step": round(line["ms_per_step"], 4),
+               "hbm_frac": round(line["step_hbm"]["frac"], 3), "merge_us": round(line["merge"]["us"], 1),
+               "assign_kernel": assign, "assign_us": round(k[assign]["avg_us"], 1) if assign else None,
+               "assign_tensor_frac": round(merge_flops(cfg) / (k[assign]["avg_us"] * 1e-6) / 1e12 / peak_tf, 4) if assign else None,
+               "kernels_us": {n: round(v["avg_us"] * v["launches_per_step"], 1) for n, v in k.items()},
+               "clocks_mhz": line["clocks"]["sm_mhz"], "reasons": line["clocks"]["reasons"]}
+        print(json.dumps(out), flush=True)
 
 
 def main():
@@ -392,6 +449,7 @@ def main():
     ap.add_argument("--merge-path", type=int, default=0, help="0 auto, 1 CUDA cores, 2 tensor cores")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="all named workloads and the batch x retention sweep")
     args = ap.parse_args()
     if args.workload.startswith("sweep:"):
         _, b, r = args.workload.split(":")
