@@ -48,6 +48,26 @@ void prof_after(cudaStream_t stream);
     VSCAN_AFTER_LAUNCH();                      \
   } while (0)
 
+// Launch with programmatic stream serialisation: the kernel may start while the previous kernel of
+// the stream is still draining; it must execute grid_dependency_wait() before it touches anything
+// that kernel produced.  Without a preceding kernel (or with an event in between) this is an
+// ordinary launch.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -73,6 +93,12 @@ inline cudaError_t allow_smem(K kernel, size_t bytes) {
 constexpr size_t kMaxDynamicSmem = 227 * 1024;
 
 // ------------------------------------------------------------------ device helpers
+// Blocks until the preceding kernel of the stream has completed and its writes are visible (no-op
+// for a kernel launched the ordinary way).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled as soon as every CTA of this grid has got here.
+__device__ __forceinline__ void grid_dependency_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <typename T>
 __device__ __forceinline__ float to_float(T v);
 template <>

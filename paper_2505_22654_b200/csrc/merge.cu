@@ -147,7 +147,7 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 // ascending token order, the tokens assigned to its slots; each warp then walks that list and adds
 // its members' rows in that order (fp32), R rows in flight.  Small CTAs keep a large group from
 // holding the resources of many finished warps.
-// dynamic shared memory: list[n_tokens] of (local slot << 24 | token)
+// dynamic shared memory: list[n_tokens] of (local slot << 24 | token), then assign[n_tokens]
 constexpr int kSlotsPerCta = 4;
 constexpr int kMeanThreads = kSlotsPerCta * 32;
 
@@ -157,7 +157,21 @@ __global__ void __launch_bounds__(kMeanThreads) group_mean_kernel(MergeParams p)
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
   const int b = blockIdx.y, s0 = blockIdx.x * kSlotsPerCta;
-  const int32_t* assign = p.assign + static_cast<size_t>(b) * p.n_tokens;
+  // all assignments of the instance -> shared memory (second half of the buffer) in one round of
+  // independent, coalesced loads; the two ordered passes below then run out of shared memory
+  int32_t* assign = reinterpret_cast<int32_t*>(list + p.n_tokens);
+  grid_dependency_wait();   // the assignments come from the kernel before this one
+  {
+    const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
+    for (int i0 = threadIdx.x; i0 < p.n_tokens; i0 += kMeanThreads * 8) {
+      int32_t v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; if (i < p.n_tokens) assign[i] = v[u]; }
+    }
+  }
+  __syncthreads();
 
   const int per = (p.n_tokens + blockDim.x - 1) / blockDim.x;
   const int lo = min(p.n_tokens, static_cast<int>(threadIdx.x) * per), hi = min(p.n_tokens, lo + per);
@@ -246,15 +260,17 @@ __global__ void __launch_bounds__(kMeanThreads) group_mean_kernel(MergeParams p)
 template <typename T>
 static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream) {
   constexpr int E = Vec16<T>::kElems;
-  const size_t smem = static_cast<size_t>(p.n_tokens) * 4 + 16;
+  const size_t smem = static_cast<size_t>(p.n_tokens) * 8 + 16;   // member list + staged assignments
   if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
   dim3 grid((p.n_kept + kSlotsPerCta - 1) / kSlotsPerCta, p.instances);
   if (p.dim / E <= 128) {
     VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4, 4>, smem));
-    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 4, 4><<<grid, kMeanThreads, smem, stream>>>(p)));
+    VSCAN_LAUNCH("group_mean", stream,
+                 (void)launch_dependent(group_mean_kernel<T, 4, 4>, grid, dim3(kMeanThreads), smem, stream, p));
   } else {
     VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8, 2>, smem));
-    VSCAN_LAUNCH("group_mean", stream, (group_mean_kernel<T, 8, 2><<<grid, kMeanThreads, smem, stream>>>(p)));
+    VSCAN_LAUNCH("group_mean", stream,
+                 (void)launch_dependent(group_mean_kernel<T, 8, 2>, grid, dim3(kMeanThreads), smem, stream, p));
   }
   return VSCAN_OK;
 }
@@ -352,8 +368,7 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   // small kernel of its own
   st = VSCAN_ERR_UNSUPPORTED;
   if (tensor) {
-    VSCAN_CUDA_TRY(cudaMemsetAsync(p.status, 0, sizeof(uint32_t), stream));
-    st = launch_assign_tensor(p, stream);
+    st = launch_assign_tensor(p, stream);   // clears the status word itself
     if (st != VSCAN_OK && (st != VSCAN_ERR_UNSUPPORTED || d->path != VSCAN_MERGE_AUTO)) return st;
   }
   if (st == VSCAN_ERR_UNSUPPORTED) {   // CUDA cores (asked for, or a shape the tensor path cannot take)

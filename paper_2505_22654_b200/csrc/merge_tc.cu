@@ -67,10 +67,13 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = sh.tmem_base;
+  grid_dependency_launch();
+  grid_dependency_wait();   // the kept list comes from the kernel before this one
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer: TMA tile + TMA row gathers
@@ -249,11 +252,13 @@ static bool plan(const MergeParams& m, Params& p) {
   p.a_stage_bytes = kTileM * kChunkK * 2;
   p.b_stage_bytes = ((p.n_pad * kChunkK * 2) + 1023) / 1024 * 1024;
   const int stage = p.a_stage_bytes + p.b_stage_bytes;
-  // two CTAs per SM when four stages fit in half the shared memory, else as many stages as fit
-  int stages = (110 * 1024) / stage;
-  if (stages < 3) stages = (215 * 1024) / stage;
+  // three CTAs per SM with three stages each when that fits (their fixed start-up and epilogue
+  // costs overlap), else two with up to four, else one CTA with as many stages as fit
+  int stages;
+  if ((73 * 1024) / stage >= 3) stages = 3;
+  else if ((110 * 1024) / stage >= 3) stages = (110 * 1024) / stage > 4 ? 4 : (110 * 1024) / stage;
+  else stages = (215 * 1024) / stage;
   if (stages > kMaxStages) stages = kMaxStages;
-  if (stages > 4 && (110 * 1024) / stage >= 4) stages = 4;
   p.stages = stages;
   return stages >= 2;
 }
@@ -296,7 +301,8 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   const size_t smem = static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
   dim3 grid((m.n_tokens + tc::kTileM - 1) / tc::kTileM, m.instances);
-  VSCAN_LAUNCH("assign_tensor", stream, tc::assign_tensor_kernel<<<grid, tc::kThreads, smem, stream>>>(map, map_b, p));
+  VSCAN_LAUNCH("assign_tensor", stream,
+               (void)launch_dependent(tc::assign_tensor_kernel, grid, dim3(tc::kThreads), smem, stream, map, map_b, p));
   return VSCAN_OK;
 }
 

@@ -41,6 +41,7 @@ __device__ __forceinline__ void copy_run(const uint4* __restrict__ src, uint4* _
 
 __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams p) {
   const int r = blockIdx.x, b = blockIdx.y;
+  grid_dependency_wait();   // the survivor list comes from the kernel before this one
   int src;
   if (r < p.n_sys) src = r;
   else if (r < p.n_sys + p.k_keep) {
@@ -181,6 +182,6 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   c.hidden_vecs = d->hidden ? static_cast<int>(d->hidden_dim * e / 16) : 0;
   c.kv_vecs = static_cast<int>(d->head_dim * e / 16);
   dim3 grid(seq_out, d->batch);
-  VSCAN_LAUNCH("compact", stream, compact_kernel<<<grid, kCompactThreads, 0, stream>>>(c));
+  VSCAN_LAUNCH("compact", stream, (void)launch_dependent(compact_kernel, grid, dim3(kCompactThreads), 0, stream, c));
   return VSCAN_OK;
 }

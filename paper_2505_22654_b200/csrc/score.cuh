@@ -38,6 +38,7 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   constexpr int E = Vec16<T>::kElems;
   constexpr int R = 4;   // key rows in flight per 8-lane group
   const int h = blockIdx.x, b = blockIdx.y;
+  grid_dependency_launch();
   if (h == 0 && b == 0 && threadIdx.x == 0 && p.status) *p.status = 0u;
   const int g = static_cast<int>((static_cast<long long>(h) * p.kv_heads) / p.q_heads);
   const T* qh = static_cast<const T*>(p.q) + (static_cast<size_t>(b) * p.q_heads + h) * p.head_dim;

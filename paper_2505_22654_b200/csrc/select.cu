@@ -52,6 +52,7 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
   uint32_t* keys_l = keys_g + p.n;
   uint8_t* taken = reinterpret_cast<uint8_t*>(keys_l + p.n);
   __shared__ SelectScratch sc;
+  grid_dependency_launch();
 
   const int b = blockIdx.x;
   if constexpr (std::is_void<T>::value) {
