@@ -13,7 +13,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) kept_inv_norm_kernel(MergeParams p) {
   constexpr int E = Vec16<T>::kElems;
   const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *p.status = 0u;
+  if (p.clear_status && blockIdx.x == 0 && b == 0 && threadIdx.x == 0) *p.status = 0u;
   if (s >= p.n_kept) return;
   int t = p.kept[static_cast<size_t>(b) * p.n_kept + s];
   t = min(max(t, 0), p.n_tokens - 1);
@@ -315,6 +315,10 @@ extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
   size_t bytes = kStatusBytes;
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256);    // inv_norm
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);  // assign
+  if (d->dtype == VSCAN_BF16 && d->n_kept > 256) {   // packed copy of the kept rows for the tensor path
+    const size_t md = d->metric ? d->metric_dim : d->dim;
+    bytes += round_up(static_cast<size_t>(d->instances) * round_up(d->n_kept, 256) * md * 2, 256);
+  }
   return bytes;
 }
 
@@ -339,9 +343,14 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   int32_t* ws_assign = reinterpret_cast<int32_t*>(
       ws + kStatusBytes + round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256));
   p.assign = d->assign ? d->assign : ws_assign;
+  p.kept_packed = (d->dtype == VSCAN_BF16 && d->n_kept > 256)
+                      ? static_cast<void*>(reinterpret_cast<char*>(ws_assign) +
+                                           round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256))
+                      : nullptr;
   p.merged = d->merged; p.counts = d->counts;
   p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
+  p.clear_status = 1;
 
   // fused kernel: one launch for the whole call
   if (d->path == VSCAN_MERGE_FUSED) {   // measured slower than the two-kernel tensor path: opt-in only
@@ -378,7 +387,8 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
     st = launch_assign_simt(d->dtype, p, stream);
     if (st != VSCAN_OK) return st;
   }
-
+  // (Cutting the batch into runs of instances small enough for L2, so that the group-mean pass of a
+  // run finds its features there, was measured slower: the smaller grids are latency-bound.)
   return d->dtype == VSCAN_F32 ? launch_group_mean<float>(p, stream)
                                : launch_group_mean<__nv_bfloat16>(p, stream);
 }

@@ -22,6 +22,7 @@ constexpr int kThreads = 192;
 
 struct Params {
   MergeParams m;
+  int b_packed;     // kept rows come from the packed copy (one tile load per stage) instead of row gathers
   int n_pad;        // kept columns per n-chunk, multiple of 16, <= 256
   int n_chunks;     // ceil(n_kept / n_pad)
   int k_chunks;     // ceil(metric_dim / 64)
@@ -40,6 +41,24 @@ struct Shared {
   int best_slot[kTileM];
   float inv_norm[2][kMaxN];
 };
+
+// Copies the kept rows of every instance into a contiguous [instance][slot][dim] buffer (slots past
+// n_kept are zero).  One warp per slot.
+__global__ void __launch_bounds__(256) pack_kept_kernel(MergeParams m, int rows_packed) {
+  const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (s >= rows_packed) return;
+  uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.kept_packed) +
+                                        (static_cast<size_t>(b) * rows_packed + s) * m.metric_dim);
+  const int vecs = m.metric_dim / 8;
+  if (s < m.n_kept) {
+    const int t = min(max(m.kept[static_cast<size_t>(b) * m.n_kept + s], 0), m.n_tokens - 1);
+    const uint4* src = reinterpret_cast<const uint4*>(
+        static_cast<const __nv_bfloat16*>(m.metric) + (static_cast<size_t>(b) * m.row_len + m.cls_offset + t) * m.metric_dim);
+    for (int v = lane; v < vecs; v += 32) st_16(dst + v, ld_nc_16(src + v));
+  } else {
+    for (int v = lane; v < vecs; v += 32) st_16(dst + v, make_uint4(0u, 0u, 0u, 0u));
+  }
+}
 
 // dynamic shared memory (1024-byte aligned): stages x [A tile 128x64 bf16 | B tile n_pad x 64 bf16]
 __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_constant__ CUtensorMap map_a,
@@ -67,7 +86,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
+  if (m.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -104,11 +123,12 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
         if (lane == 0) {
           mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes + p.n_pad * 128);
           tma_load_3d(at, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
+          if (p.b_packed) tma_load_3d(at + p.a_stage_bytes, &map_b, &sh.full[s], kc * kChunkK, nc * p.n_pad, b);
         }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           const int g = lane + 32 * i;
-          if (g < groups)
+          if (g < groups && !p.b_packed)
             tma_gather4(at + p.a_stage_bytes + g * 512, &map_b, &sh.full[s], kc * kChunkK, rows[i][0], rows[i][1],
                         rows[i][2], rows[i][3]);
         }
@@ -243,6 +263,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
 // ---------------------------------------------------------------------------- host side
 static bool plan(const MergeParams& m, Params& p) {
   p.m = m;
+  p.b_packed = (m.n_kept > kMaxN && m.kept_packed != nullptr) ? 1 : 0;
   const int n16 = (m.n_kept + 15) / 16 * 16;
   p.n_pad = n16 <= kMaxN ? n16 : kMaxN;
   p.n_chunks = (m.n_kept + p.n_pad - 1) / p.n_pad;
@@ -294,10 +315,25 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
                                 static_cast<cuuint64_t>(m.row_len) * static_cast<cuuint64_t>(m.instances)};
   const cuuint64_t strides_b[1] = {static_cast<cuuint64_t>(m.metric_dim) * 2};
   const cuuint32_t box_b[2] = {tc::kChunkK, 1};
-  r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(m.metric), dims_b, strides_b, box_b, elem,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (p.b_packed) {
+    // large kept sets: the rows were packed into [instance][slot][dim] beforehand, one tile load per stage
+    const cuuint64_t rows_packed = static_cast<cuuint64_t>(p.n_chunks) * p.n_pad;
+    const cuuint64_t dims_p[3] = {static_cast<cuuint64_t>(m.metric_dim), rows_packed, static_cast<cuuint64_t>(m.instances)};
+    const cuuint64_t strides_p[2] = {static_cast<cuuint64_t>(m.metric_dim) * 2, rows_packed * m.metric_dim * 2};
+    const cuuint32_t box_p[3] = {tc::kChunkK, static_cast<cuuint32_t>(p.n_pad), 1};
+    r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m.kept_packed, dims_p, strides_p, box_p, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  } else {
+    r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(m.metric), dims_b, strides_b, box_b, elem,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }
   if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
+  if (p.b_packed) {
+    dim3 pgrid((static_cast<unsigned>(p.n_chunks) * p.n_pad + 7) / 8, m.instances);
+    VSCAN_LAUNCH("pack_kept", stream, tc::pack_kept_kernel<<<pgrid, 256, 0, stream>>>(m, p.n_chunks * p.n_pad));
+  }
   const size_t smem = static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
   dim3 grid((m.n_tokens + tc::kTileM - 1) / tc::kTileM, m.instances);

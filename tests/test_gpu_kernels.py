@@ -180,7 +180,7 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
             vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_FUSED)
         assert e.value.status == 2       # more kept tokens than one accumulator holds: not this path
         return
-    ws = vs.Workspace(1 << 20)
+    ws = vs.Workspace(8 << 20)
     merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
                                             want_counts=True, workspace=ws,
                                             path=vs.MERGE_TENSOR if path == "tensor" else vs.MERGE_FUSED)
