@@ -47,6 +47,7 @@ def algorithmic_bytes(cfg) -> dict:
         "compact": B * 2 * cfg.S_out * (cfg.Dh * e + 2 * cfg.Hkv * cfg.d * e + cfg.pos_planes * 4),
     }
     row["score_select"] = 2 * I * cfg.H * cfg.L * e + I * (2 * cfg.N * 4 + cfg.K1 * 4)   # fused Eq. 2 + Eq. 3
+    row["prune_fused"] = row["qk_softmax"] + row["prune_topk"] + row["compact"]   # Stage 2 in one launch
     row["step"] = 2 * row["row_mean"] + row["select"] + row["merge"] + row["qk_softmax"] + \
         row["prune_topk"] + row["compact"]
     return row

@@ -143,16 +143,15 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 }
 
 // ------------------------------------------------------------------ group means
-// One CTA per (group of 4 slots, instance); warp w owns slot s0 + w.  The CTA first lists, in
+// One CTA per (group of slots, instance), one warp per slot: 4 slots per CTA for short instances, 16
+// for long ones (the list-building prologue is O(n_tokens) per CTA); warp w owns slot s0 + w.  The CTA first lists, in
 // ascending token order, the tokens assigned to its slots; each warp then walks that list and adds
 // its members' rows in that order (fp32), R rows in flight.  Small CTAs keep a large group from
 // holding the resources of many finished warps.
 // dynamic shared memory: list[n_tokens] of (local slot << 24 | token), then assign[n_tokens]
-constexpr int kSlotsPerCta = 4;
-constexpr int kMeanThreads = kSlotsPerCta * 32;
-
-template <typename T, int VPL, int R>
-__global__ void __launch_bounds__(kMeanThreads) group_mean_kernel(MergeParams p) {
+template <typename T, int VPL, int R, int kSlotsPerCta>
+__global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergeParams p) {
+  constexpr int kMeanThreads = kSlotsPerCta * 32;
   constexpr int E = Vec16<T>::kElems;
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
@@ -257,22 +256,25 @@ __global__ void __launch_bounds__(kMeanThreads) group_mean_kernel(MergeParams p)
   }
 }
 
+template <typename T, int VPL, int R, int SLOTS>
+static vscan_status launch_group_mean_as(const MergeParams& p, size_t smem, cudaStream_t stream) {
+  dim3 grid((p.n_kept + SLOTS - 1) / SLOTS, p.instances);
+  VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, VPL, R, SLOTS>, smem));
+  VSCAN_LAUNCH("group_mean", stream,
+               (void)launch_dependent(group_mean_kernel<T, VPL, R, SLOTS>, grid, dim3(SLOTS * 32), smem, stream, p));
+  return VSCAN_OK;
+}
+
 template <typename T>
 static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream) {
   constexpr int E = Vec16<T>::kElems;
   const size_t smem = static_cast<size_t>(p.n_tokens) * 8 + 16;   // member list + staged assignments
   if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
-  dim3 grid((p.n_kept + kSlotsPerCta - 1) / kSlotsPerCta, p.instances);
-  if (p.dim / E <= 128) {
-    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 4, 4>, smem));
-    VSCAN_LAUNCH("group_mean", stream,
-                 (void)launch_dependent(group_mean_kernel<T, 4, 4>, grid, dim3(kMeanThreads), smem, stream, p));
-  } else {
-    VSCAN_CUDA_TRY(allow_smem(group_mean_kernel<T, 8, 2>, smem));
-    VSCAN_LAUNCH("group_mean", stream,
-                 (void)launch_dependent(group_mean_kernel<T, 8, 2>, grid, dim3(kMeanThreads), smem, stream, p));
-  }
-  return VSCAN_OK;
+  const bool wide = p.dim / E > 128, long_instance = p.n_tokens > 2048;
+  if (!wide && !long_instance) return launch_group_mean_as<T, 4, 4, 4>(p, smem, stream);
+  if (!wide) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
+  if (!long_instance) return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
+  return launch_group_mean_as<T, 8, 2, 16>(p, smem, stream);
 }
 
 }  // namespace vscan

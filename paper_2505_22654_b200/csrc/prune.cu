@@ -22,36 +22,37 @@ struct CompactParams {
 constexpr int kCompactThreads = 256;
 constexpr int kCompactUnroll = 4;
 
+template <int THREADS>
 __device__ __forceinline__ void copy_run(const uint4* __restrict__ src, uint4* __restrict__ dst, int n) {
   // n pieces, contiguous on both sides
-  for (int i0 = threadIdx.x; i0 < n; i0 += kCompactThreads * kCompactUnroll) {
+  for (int i0 = threadIdx.x; i0 < n; i0 += THREADS * kCompactUnroll) {
     uint4 r[kCompactUnroll];
 #pragma unroll
     for (int u = 0; u < kCompactUnroll; ++u) {
-      int i = i0 + u * kCompactThreads;
+      int i = i0 + u * THREADS;
       if (i < n) r[u] = ld_nc_16(src + i);
     }
 #pragma unroll
     for (int u = 0; u < kCompactUnroll; ++u) {
-      int i = i0 + u * kCompactThreads;
+      int i = i0 + u * THREADS;
       if (i < n) st_16(dst + i, r[u]);
     }
   }
 }
 
-__global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams p) {
-  const int r = blockIdx.x, b = blockIdx.y;
-  grid_dependency_wait();   // the survivor list comes from the kernel before this one
+// Moves output row r of sequence b: hidden row, the kv_heads rows of K and of V, position ids.
+template <int THREADS>
+__device__ __forceinline__ void compact_row(const CompactParams& p, const int r, const int b) {
   int src;
   if (r < p.n_sys) src = r;
   else if (r < p.n_sys + p.k_keep) {
-    int kv = p.kept_vis[static_cast<size_t>(b) * p.k_keep + (r - p.n_sys)];
+    int kv = __ldcg(p.kept_vis + static_cast<size_t>(b) * p.k_keep + (r - p.n_sys));
     kv = min(max(kv, 0), p.n_vis - 1);
     src = p.n_sys + kv;
   } else src = r + (p.n_vis - p.k_keep);
 
   if (p.hidden) {
-    copy_run(p.hidden + (static_cast<size_t>(b) * p.seq_len + src) * p.hidden_vecs,
+    copy_run<THREADS>(p.hidden + (static_cast<size_t>(b) * p.seq_len + src) * p.hidden_vecs,
              p.hidden_out + (static_cast<size_t>(b) * p.seq_out + r) * p.hidden_vecs, p.hidden_vecs);
   }
   // K and V: kv_heads rows of kv_vecs pieces, strided by the sequence length
@@ -59,12 +60,12 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
   const size_t src_head = static_cast<size_t>(p.seq_len) * p.kv_vecs, dst_head = static_cast<size_t>(p.seq_out) * p.kv_vecs;
   const size_t src0 = (static_cast<size_t>(b) * p.kv_heads * p.seq_len + src) * p.kv_vecs;
   const size_t dst0 = (static_cast<size_t>(b) * p.kv_heads * p.seq_out + r) * p.kv_vecs;
-  for (int i0 = threadIdx.x; i0 < total; i0 += kCompactThreads * kCompactUnroll) {
+  for (int i0 = threadIdx.x; i0 < total; i0 += THREADS * kCompactUnroll) {
     uint4 rk[kCompactUnroll], rv[kCompactUnroll];
     size_t so[kCompactUnroll], dof[kCompactUnroll];
 #pragma unroll
     for (int u = 0; u < kCompactUnroll; ++u) {
-      int i = i0 + u * kCompactThreads;
+      int i = i0 + u * THREADS;
       if (i < total) {
         int head = i / p.kv_vecs, vec = i - head * p.kv_vecs;
         so[u] = src0 + head * src_head + vec;
@@ -75,7 +76,7 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
     }
 #pragma unroll
     for (int u = 0; u < kCompactUnroll; ++u) {
-      int i = i0 + u * kCompactThreads;
+      int i = i0 + u * THREADS;
       if (i < total) {
         st_16(p.k_out + dof[u], rk[u]);
         if (p.v) st_16(p.v_out + dof[u], rv[u]);
@@ -87,6 +88,79 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
     p.pos_out[(static_cast<size_t>(pl) * p.batch + b) * p.seq_out + r] =
         p.pos[(static_cast<size_t>(pl) * p.batch + b) * p.seq_len + src];
   }
+}
+
+__global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams p) {
+  grid_dependency_wait();   // the survivor list comes from the kernel before this one
+  compact_row<kCompactThreads>(p, blockIdx.x, blockIdx.y);
+}
+
+// Score, top-k and compaction of Stage 2 in ONE launch.  The first n_score CTAs are the (head,
+// sequence) scoring CTAs of qk_softmax_role; the CTAs after them each move one output row.  Rows of
+// the system and text spans do not depend on the selection and are moved at once (they come first
+// in block order); a row of the visual span waits, with a bound, until the scoring CTA that finished
+// its sequence last has published the survivor list.  Blocks are dispatched in index order, so
+// every scoring CTA is running or done before a waiting CTA can occupy a slot.
+constexpr int kPruneThreads = 128;
+constexpr unsigned kReadySpinLimit = 1u << 22;
+
+template <typename T, int VPS>
+__global__ void __launch_bounds__(kPruneThreads) prune_fused_kernel(QkParams q, CompactParams c, int n_score) {
+  extern __shared__ __align__(16) float smem_f[];
+  const int blk = blockIdx.x;
+  if (blk < n_score) {
+    qk_softmax_role<T, VPS>(q, blk % q.q_heads, blk / q.q_heads, smem_f);
+    return;
+  }
+  int idx = blk - n_score;
+  const int fixed_rows = c.seq_out - c.k_keep;           // system + text rows per sequence
+  int r, b;
+  bool dependent;
+  if (idx < c.batch * fixed_rows) {
+    b = idx / fixed_rows;
+    const int i = idx - b * fixed_rows;
+    r = i < c.n_sys ? i : i + c.k_keep;
+    dependent = false;
+  } else {
+    idx -= c.batch * fixed_rows;
+    b = idx / c.k_keep;
+    r = c.n_sys + (idx - b * c.k_keep);
+    dependent = true;
+  }
+  if (dependent) {
+    __shared__ int ok;
+    if (threadIdx.x == 0) {
+      unsigned spins = 0;
+      const volatile int* flag = q.ready + b;
+      while (*flag == 0 && spins < kReadySpinLimit) { __nanosleep(100); ++spins; }
+      ok = *flag != 0;
+      if (!ok && q.status) atomicExch(q.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+      __threadfence();
+    }
+    __syncthreads();
+    if (!ok) return;
+  }
+  compact_row<kPruneThreads>(c, r, b);
+}
+
+template <typename T>
+static vscan_status launch_prune_fused(const QkParams& q, const CompactParams& c, size_t smem, cudaStream_t stream) {
+  constexpr int E = Vec16<T>::kElems;
+  const int n_score = c.batch * q.q_heads;
+  const unsigned blocks = static_cast<unsigned>(n_score) + static_cast<unsigned>(c.batch) * c.seq_out;
+  const int vecs = q.head_dim / E;
+#define VSCAN_PRUNE_CASE(VPS)                                                                                  \
+  do {                                                                                                         \
+    VSCAN_CUDA_TRY(allow_smem(prune_fused_kernel<T, VPS>, smem));                                              \
+    VSCAN_LAUNCH("prune_fused", stream,                                                                        \
+                 (prune_fused_kernel<T, VPS><<<blocks, kPruneThreads, smem, stream>>>(q, c, n_score)));        \
+    return VSCAN_OK;                                                                                           \
+  } while (0)
+  if (vecs == 16) VSCAN_PRUNE_CASE(2);
+  if (vecs == 32) VSCAN_PRUNE_CASE(4);
+  if (vecs == 8) VSCAN_PRUNE_CASE(1);
+  VSCAN_PRUNE_CASE(0);
+#undef VSCAN_PRUNE_CASE
 }
 
 }  // namespace vscan
@@ -108,7 +182,7 @@ static vscan_status validate_prune(const vscan_prune_desc* d) {
   const size_t e = dtype_bytes(d->dtype);
   if (d->hidden && (d->hidden_dim <= 0 || (d->hidden_dim * e) % 16)) return VSCAN_ERR_INVALID_ARG;
   if (d->pos_ids && d->pos_planes <= 0) return VSCAN_ERR_INVALID_ARG;
-  if (d->pos_ids && d->pos_planes > vscan::kCompactThreads) return VSCAN_ERR_UNSUPPORTED;
+  if (d->pos_ids && d->pos_planes > vscan::kPruneThreads) return VSCAN_ERR_UNSUPPORTED;
   if (d->n_vis > 16384) return VSCAN_ERR_UNSUPPORTED;
   const void* ptrs[] = {d->q_last, d->k, d->v, d->hidden, d->pos_ids, d->kept_vis, d->hidden_out,
                         d->k_out, d->v_out, d->pos_out, d->scores};
@@ -134,7 +208,7 @@ static vscan_status validate_prune(const vscan_prune_desc* d) {
 
 extern "C" size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* d) {
   if (!d || d->batch <= 0 || d->q_heads <= 0 || d->n_vis <= 0) return kStatusBytes;
-  return kStatusBytes + round_up(static_cast<size_t>(d->batch) * sizeof(int), 256) +
+  return kStatusBytes + round_up(2 * static_cast<size_t>(d->batch) * sizeof(int), 256) +
          round_up(static_cast<size_t>(d->batch) * d->q_heads * d->n_vis * sizeof(float), 256);
 }
 
@@ -148,28 +222,9 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   const size_t need = vscan_llm_prune_workspace_bytes(d);
   if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
   const int seq_len = d->n_sys + d->n_vis + d->n_txt, seq_out = seq_len - d->n_vis + d->k_keep;
-  // workspace: status word | per-sequence arrival counters | per-head probabilities
+  // workspace: status word | per-sequence arrival counters, per-sequence ready flags | per-head probabilities
   char* ws = static_cast<char*>(workspace);
-  const size_t counter_bytes = round_up(static_cast<size_t>(d->batch) * sizeof(int), 256);
-
-  if (d->n_vis > 0) {
-    QkParams p;
-    p.q = d->q_last; p.k = d->k; p.status = static_cast<uint32_t*>(workspace);
-    p.counters = reinterpret_cast<int*>(ws + kStatusBytes);
-    p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes);
-    p.scores = d->scores; p.kept = d->kept_vis; p.k_keep = d->k_keep;
-    p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = seq_len; p.head_dim = d->head_dim;
-    p.span_begin = d->n_sys; p.span_len = d->n_vis; p.scale = d->scale;
-    if (d->softmax_span == VSCAN_SPAN_ONLY) { p.soft_lo = d->n_sys; p.soft_n = d->n_vis; }
-    else { p.soft_lo = 0; p.soft_n = seq_len; }
-    // score and top-k in one launch: the last CTA of each sequence reduces over the heads and selects
-    VSCAN_CUDA_TRY(cudaMemsetAsync(p.counters, 0, counter_bytes, stream));
-    st = launch_qk_softmax(d->dtype, p, d->batch, stream);
-    if (st != VSCAN_OK) return st;
-  } else {
-    VSCAN_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, stream));
-  }
-  if (seq_out == 0) return VSCAN_OK;
+  const size_t counter_bytes = round_up(2 * static_cast<size_t>(d->batch) * sizeof(int), 256);
   const size_t e = dtype_bytes(d->dtype);
   CompactParams c;
   c.kept_vis = d->kept_vis;
@@ -181,6 +236,37 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   c.n_sys = d->n_sys; c.n_vis = d->n_vis; c.k_keep = d->k_keep; c.pos_planes = d->pos_planes;
   c.hidden_vecs = d->hidden ? static_cast<int>(d->hidden_dim * e / 16) : 0;
   c.kv_vecs = static_cast<int>(d->head_dim * e / 16);
+
+  bool fused = false;
+  if (d->n_vis > 0) {
+    QkParams p;
+    p.q = d->q_last; p.k = d->k; p.status = static_cast<uint32_t*>(workspace);
+    p.counters = reinterpret_cast<int*>(ws + kStatusBytes);
+    p.ready = p.counters + d->batch;
+    p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes);
+    p.scores = d->scores; p.kept = d->kept_vis; p.k_keep = d->k_keep;
+    p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = seq_len; p.head_dim = d->head_dim;
+    p.span_begin = d->n_sys; p.span_len = d->n_vis; p.scale = d->scale;
+    if (d->softmax_span == VSCAN_SPAN_ONLY) { p.soft_lo = d->n_sys; p.soft_n = d->n_vis; }
+    else { p.soft_lo = 0; p.soft_n = seq_len; }
+    VSCAN_CUDA_TRY(cudaMemsetAsync(p.counters, 0, counter_bytes, stream));
+    // one launch for score, top-k and compaction when the top-k fits the 128-thread scoring CTAs
+    const long long blocks = 1ll * d->batch * d->q_heads + 1ll * d->batch * seq_out;
+    const size_t smem = qk_smem_bytes(p.head_dim, p.soft_n);
+    if (d->n_vis <= 8192 && seq_out > 0 && blocks < (1ll << 31) && smem <= kMaxDynamicSmem) {
+      st = d->dtype == VSCAN_F32 ? launch_prune_fused<float>(p, c, smem, stream)
+                                 : launch_prune_fused<__nv_bfloat16>(p, c, smem, stream);
+      if (st != VSCAN_OK) return st;
+      fused = true;
+    } else {
+      p.ready = nullptr;
+      st = launch_qk_softmax(d->dtype, p, d->batch, stream);
+      if (st != VSCAN_OK) return st;
+    }
+  } else {
+    VSCAN_CUDA_TRY(cudaMemsetAsync(workspace, 0, kStatusBytes, stream));
+  }
+  if (fused || seq_out == 0) return VSCAN_OK;
   dim3 grid(seq_out, d->batch);
   VSCAN_LAUNCH("compact", stream, (void)launch_dependent(compact_kernel, grid, dim3(kCompactThreads), 0, stream, c));
   return VSCAN_OK;

@@ -19,6 +19,7 @@ struct QkParams {
   float* scores = nullptr;     // [batch][span_len] head mean (optional)
   int32_t* kept = nullptr;     // [batch][k_keep] top-k of the head mean, ascending (optional)
   int k_keep = 0;
+  int* ready = nullptr;        // [batch] set to 1 once `kept` of the sequence is written (optional)
 };
 
 // One CTA per (query head, sequence).  Dynamic shared memory: q[head_dim] floats | z[soft_n] floats.
@@ -28,8 +29,7 @@ struct QkParams {
 // With `counters` set, the CTA that finishes a sequence last sums the per-head probabilities in head
 // order (the same fixed order whichever CTA it is), writes the head mean and/or its exact top-k.
 template <typename T, int VPS>
-__global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
-  extern __shared__ __align__(16) float smem_f[];
+__device__ __forceinline__ void qk_softmax_role(const QkParams& p, const int h, const int b, float* smem_f) {
   float* qs = smem_f;
   float* z = smem_f + p.head_dim;
   __shared__ float red[33];
@@ -37,8 +37,6 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   __shared__ int is_last;
   constexpr int E = Vec16<T>::kElems;
   constexpr int R = 4;   // key rows in flight per 8-lane group
-  const int h = blockIdx.x, b = blockIdx.y;
-  grid_dependency_launch();
   if (h == 0 && b == 0 && threadIdx.x == 0 && p.status) *p.status = 0u;
   const int g = static_cast<int>((static_cast<long long>(h) * p.kv_heads) / p.q_heads);
   const T* qh = static_cast<const T*>(p.q) + (static_cast<size_t>(b) * p.q_heads + h) * p.head_dim;
@@ -171,6 +169,18 @@ __global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
   __syncthreads();
   if (p.kept && p.k_keep > 0)
     block_topk_emit(keys, p.span_len, p.k_keep, sc, p.kept + static_cast<size_t>(b) * p.k_keep);
+  if (p.ready) {   // publish: the survivor list of sequence b is complete
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) atomicExch(&p.ready[b], 1);
+  }
+}
+
+template <typename T, int VPS>
+__global__ void __launch_bounds__(256) qk_softmax_kernel(QkParams p) {
+  extern __shared__ __align__(16) float smem_f[];
+  grid_dependency_launch();
+  qk_softmax_role<T, VPS>(p, blockIdx.x, blockIdx.y, smem_f);
 }
 
 inline size_t qk_smem_bytes(int head_dim, int soft_n) {
