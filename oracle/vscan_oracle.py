@@ -47,6 +47,20 @@ def score_row(attn: np.ndarray, cls_offset: int) -> np.ndarray:
     return total / H
 
 
+def cls_attention_rows(q_cls: np.ndarray, k: np.ndarray, scale: float) -> np.ndarray:
+    """Eq. 1 for one instance: S^h = Softmax(scale * Q_cls^h K^h^T) over all L keys of the layer
+    ([CLS] itself included), one row per head.  q_cls: [H, d], k: [H, L, d].  Returns [H, L]."""
+    q = np.asarray(q_cls, dtype=np.float64)
+    kk = np.asarray(k, dtype=np.float64)
+    rows = np.empty(kk.shape[:2])
+    for h in range(q.shape[0]):
+        z = scale * (kk[h] @ q[h])
+        z = z - z.max()
+        e = np.exp(z)
+        rows[h] = e / e.sum()
+    return rows
+
+
 def received_attention(probs: np.ndarray) -> np.ndarray:
     """Sec. 4.1 (text after Eq. 2): for an encoder without [CLS], the score source is the average
     attention each token receives from the *other* tokens.

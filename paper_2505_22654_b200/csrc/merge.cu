@@ -172,7 +172,8 @@ __global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergePara
   }
   __syncthreads();
 
-  const int per = (p.n_tokens + blockDim.x - 1) / blockDim.x;
+  // contiguous run of tokens per thread; an odd run length keeps the threads of a warp on different banks
+  const int per = ((p.n_tokens + blockDim.x - 1) / blockDim.x) | 1;
   const int lo = min(p.n_tokens, static_cast<int>(threadIdx.x) * per), hi = min(p.n_tokens, lo + per);
   int mine = 0;
   for (int i = lo; i < hi; ++i) {

@@ -227,6 +227,24 @@ def test_score_qk(dtype, span, B, Hq, Hkv, S, d, b0, n):
         np.testing.assert_allclose(got.sum(-1), 1.0, atol=1e-5)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_cls_scores_from_q_and_k_eq1_eq2(dtype):
+    """Eq. 1 + Eq. 2 without materialised attention rows: the QK mode with the [CLS] query of an encoder
+    layer (softmax over all keys, span = the patches) gives the same scores as the head mean of the
+    Eq. 1 rows, and feeds the selection directly."""
+    B, H, N, d = 3, 16, 576, 64
+    q = round_to_dtype(RNG.standard_normal((B, H, d)).astype(np.float32), dtype)
+    k = round_to_dtype(RNG.standard_normal((B, H, N + 1, d)).astype(np.float32), dtype)
+    scale = float(np.float32(d ** -0.5))
+    got = vs.vscan_score_qk(dev(q, dtype), dev(k, dtype), 1, N, scale, vs.SPAN_FULL)
+    ref = np.stack([vo.score_row(vo.cls_attention_rows(q[b], k[b], scale), 1) for b in range(B)])
+    assert np.abs(got.cpu().numpy() - ref).max() <= TOL_SCORE
+    kept = vs.vscan_select_global_local(got, got, 1, 24, 24, 6, 6, 2, 32).cpu().numpy()
+    g32 = got.cpu().numpy()
+    for b in range(B):
+        np.testing.assert_array_equal(kept[b], vo.select_global_local(g32[b], g32[b], 1, 24, 24, 6, 6, 2, 32)[0])
+
+
 # ------------------------------------------------------------------ vscan_llm_prune
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("span", [vo.SPAN_ONLY, vo.SPAN_FULL])

@@ -75,6 +75,21 @@ def test_score_row_uniform_and_linear():
     np.testing.assert_allclose(vo.score_row(attn, 1), 1.5 * ramp[1:])
 
 
+def test_cls_attention_rows_eq1():
+    # planted distribution: q = e_0 / scale, K_j = log(p_j) e_0  ->  the softmax returns p
+    H, L, d, scale = 3, 6, 4, 0.5
+    p = RNG.random((H, L)); p /= p.sum(1, keepdims=True)
+    q = np.zeros((H, d)); q[:, 0] = 1 / scale
+    k = np.zeros((H, L, d)); k[:, :, 0] = np.log(p)
+    np.testing.assert_allclose(vo.cls_attention_rows(q, k, scale), p, atol=1e-14)
+    # library special case, and Eq. 1 -> Eq. 2 equals the Eq. 5 form with the softmax over all keys
+    q2 = RNG.standard_normal((H, d)); k2 = RNG.standard_normal((H, L, d))
+    ref = torch.softmax(torch.from_numpy(0.7 * np.einsum("hd,hld->hl", q2, k2)), dim=-1).numpy()
+    rows = vo.cls_attention_rows(q2, k2, 0.7)
+    np.testing.assert_allclose(rows, ref, atol=1e-15)
+    np.testing.assert_allclose(vo.score_row(rows, 1), vo.score_qk(q2, k2, 1, L - 1, 0.7, vo.SPAN_FULL), atol=1e-15)
+
+
 def test_received_attention_excludes_self():
     # Two heads, three tokens.  Head 0: every query attends only to itself -> receives 0 from
     # others.  Head 1: every query attends uniformly -> each token receives 1/3 from each of the
