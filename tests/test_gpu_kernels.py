@@ -265,6 +265,31 @@ def test_llm_prune_small_planted(dtype, span):
         np.testing.assert_array_equal(out["pos"][:, b].cpu().numpy(), case["pos_ids"][:, b][:, rows])
 
 
+def test_multi_turn_reselection_from_the_same_pool():
+    """App. B "multi-turn conversations": a new question re-scores and re-selects from the existing
+    token pool.  The library is stateless, so this is a second call with the new last-token query on
+    the same keys; each turn must match the oracle on its own."""
+    cfg = small_cfg("bf16")
+    base = stage2_case(cfg)
+    kd, vd, hd, pd = dev(base["k"], "bf16"), dev(base["v"], "bf16"), dev(base["hidden"], "bf16"), dev(base["pos_ids"])
+    ws = vs.Workspace(1 << 20)
+    kept_turns = []
+    for turn in range(3):
+        q = round_to_dtype(RNG.standard_normal(base["q_last"].shape).astype(np.float32) * 4, "bf16")
+        out = vs.vscan_llm_prune(dev(q, "bf16"), kd, vd, hd, pd, cfg.n_sys, cfg.n_vis, cfg.n_txt, cfg.k2, base["scale"],
+                                 want_scores=True, workspace=ws)
+        s32 = out["scores"].cpu().numpy()
+        for b in range(cfg.B):
+            ref = vo.score_qk(q[b], base["k"][b], cfg.n_sys, cfg.n_vis, base["scale"])
+            assert np.abs(s32[b] - ref).max() <= TOL_SCORE
+            # selection is decided on the kernel's fp32 scores: feed exactly those to the oracle
+            np.testing.assert_array_equal(out["kept_vis"][b].cpu().numpy(), vo.topk_lowest_index(s32[b], cfg.k2))
+            rows = vo.compaction_rows(cfg.n_sys, cfg.n_vis, cfg.n_txt, out["kept_vis"][b].cpu().numpy())
+            np.testing.assert_array_equal(out["hidden"][b].float().cpu().numpy(), base["hidden"][b][rows])
+        kept_turns.append(out["kept_vis"].cpu().numpy().copy())
+    assert any(not np.array_equal(kept_turns[0], k) for k in kept_turns[1:])     # different questions, different sets
+
+
 @pytest.mark.parametrize("k_keep,n_sys,n_txt", [(0, 3, 4), (20, 3, 4), (7, 0, 0), (20, 0, 5), (1, 2, 0)])
 def test_llm_prune_edges(k_keep, n_sys, n_txt):
     n_vis, Hq, Hkv, d, Dh, B = 20, 4, 2, 16, 24, 2

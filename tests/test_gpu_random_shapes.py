@@ -1,0 +1,90 @@
+"""Seeded random shapes: every call against the oracle on small odd sizes (dims that are not multiples
+of the tile sizes, windows of every aspect, kept counts from 1 to all, grouped heads).  Margins are
+planted where a floating-point decision picks an index; scores are compared through the kernel's own
+fp32 values where they are not."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2505_22654_b200 as vs
+from oracle import plant
+from oracle import vscan_oracle as vo
+from synth import CONFIGS, round_to_dtype
+
+from helpers import TOL_SCORE, check_merged, dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _cfg(dtype, **kw):
+    return CONFIGS[2].with_(name="rand", config_id=77, dtype=dtype, **kw)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_stage1(seed):
+    rng = np.random.default_rng(1000 + seed)
+    dtype = ["f32", "bf16"][seed % 2]
+    F = int(rng.integers(1, 3)); wh, ww = int(rng.integers(1, 5)), int(rng.integers(1, 5))
+    Gh, Gw = wh * int(rng.integers(1, 5)), ww * int(rng.integers(1, 5))
+    N = F * Gh * Gw
+    W = F * (Gh // wh) * (Gw // ww)
+    k_w = int(rng.integers(0, wh * ww + 1))
+    k_g = int(rng.integers(0, N - W * k_w + 1))
+    if W * k_w + k_g == 0:
+        k_g = 1
+    c, H, B = int(rng.integers(0, 2)), int(rng.integers(1, 20)), int(rng.integers(1, 4))
+    D = 8 * int(rng.integers(1, 40))
+    cfg = _cfg(dtype, B=B, C=1, frames=F, grid_h=Gh, grid_w=Gw, win_h=wh, win_w=ww, k_w=k_w, k_g=k_g, cls=c, H=H, D=D)
+    ag = round_to_dtype(rng.random((B, H, N + c)).astype(np.float32) / max(N, 1), dtype)
+    al = round_to_dtype(rng.random((B, H, N + c)).astype(np.float32) / max(N, 1), dtype)
+    plant.plant_stage1_scores(cfg, ag, al)
+    kept = vs.vscan_score_select(dev(ag, dtype), dev(al, dtype), c, F, Gh, Gw, wh, ww, k_w, k_g)
+    ref = np.stack([vo.select_global_local(vo.score_row(ag[b], c), vo.score_row(al[b], c), F, Gh, Gw, wh, ww, k_w, k_g)[0]
+                    for b in range(B)])
+    np.testing.assert_array_equal(kept.cpu().numpy(), ref)
+    # un-fused calls give the same list
+    sg, sl = vs.vscan_score_row(dev(ag, dtype), c), vs.vscan_score_row(dev(al, dtype), c)
+    kept2 = vs.vscan_select_global_local(sg, sl, F, Gh, Gw, wh, ww, k_w, k_g)
+    assert torch.equal(kept, kept2)
+    # merge on those kept tokens, every path the dtype allows
+    x = round_to_dtype(rng.standard_normal((B, N + c, D)).astype(np.float32), dtype)
+    plant.plant_merge(cfg, x, ref)
+    paths = [vs.MERGE_AUTO, vs.MERGE_SIMT] + ([vs.MERGE_TENSOR, vs.MERGE_FUSED] if dtype == "bf16" and ref.shape[1] <= 256 else [])
+    for path in paths:
+        merged, assign, counts = vs.vscan_merge(dev(x, dtype), c, kept, path=path, want_assign=True, want_counts=True)
+        for b in range(B):
+            m, a, cn = vo.merge(x[b], c, ref[b])
+            np.testing.assert_array_equal(assign[b].cpu().numpy(), a, err_msg=f"path {path}")
+            np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
+            check_merged(merged[b], m, dtype)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_stage2(seed):
+    rng = np.random.default_rng(2000 + seed)
+    dtype = ["f32", "bf16"][seed % 2]
+    Hkv = int(rng.integers(1, 5)); Hq = Hkv * int(rng.integers(1, 5))
+    d = 8 * int(rng.integers(1, 17)); Dh = 8 * int(rng.integers(1, 33))
+    n_sys, n_vis, n_txt = int(rng.integers(0, 6)), int(rng.integers(1, 200)), int(rng.integers(0, 9))
+    k_keep = int(rng.integers(0, n_vis + 1))
+    B, P = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+    span = [vo.SPAN_ONLY, vo.SPAN_FULL][seed % 3 == 0]
+    S = n_sys + n_vis + n_txt
+    cfg = _cfg(dtype, B=B, n_sys=n_sys, n_txt=n_txt, Hq=Hq, Hkv=Hkv, d=d, Dh=Dh, k2=k_keep, pos_planes=P)
+    q = round_to_dtype(rng.standard_normal((B, Hq, d)).astype(np.float32), dtype)
+    k = round_to_dtype(rng.standard_normal((B, Hkv, S, d)).astype(np.float32), dtype)
+    v = round_to_dtype(rng.standard_normal((B, Hkv, S, d)).astype(np.float32), dtype)
+    h = round_to_dtype(rng.standard_normal((B, S, Dh)).astype(np.float32), dtype)
+    pos = rng.integers(0, 1000, (P, B, S)).astype(np.int32)
+    scale = float(np.float32(d ** -0.5))
+    plant.plant_stage2(cfg, q, k, scale, span, n_vis=n_vis, k_keep=k_keep)
+    out = vs.vscan_llm_prune(dev(q, dtype), dev(k, dtype), dev(v, dtype), dev(h, dtype), dev(pos), n_sys, n_vis, n_txt,
+                             k_keep, scale, span, want_scores=True)
+    for b in range(B):
+        o = vo.llm_prune(q[b], k[b], v[b], h[b], pos[:, b], n_sys, n_vis, n_txt, k_keep, scale, span)
+        assert np.abs(out["scores"][b].cpu().numpy() - o["scores"]).max() <= TOL_SCORE
+        np.testing.assert_array_equal(out["kept_vis"][b].cpu().numpy(), o["kept_vis"])
+        np.testing.assert_array_equal(out["hidden"][b].float().cpu().numpy(), o["hidden"])
+        np.testing.assert_array_equal(out["k"][b].float().cpu().numpy(), o["k"])
+        np.testing.assert_array_equal(out["v"][b].float().cpu().numpy(), o["v"])
+        np.testing.assert_array_equal(out["pos"][:, b].cpu().numpy(), o["pos"])
