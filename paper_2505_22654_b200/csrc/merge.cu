@@ -272,10 +272,11 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   const size_t smem = static_cast<size_t>(p.n_tokens) * 8 + 16;   // member list + staged assignments
   if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
   const bool wide = p.dim / E > 128, long_instance = p.n_tokens > 2048;
-  if (!wide && !long_instance) return launch_group_mean_as<T, 4, 4, 4>(p, smem, stream);
-  if (!wide) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
-  if (!long_instance) return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
-  return launch_group_mean_as<T, 8, 2, 16>(p, smem, stream);
+  // 512-thread CTAs have 128 registers per thread: wide rows are then summed in two column passes
+  // (4 pieces per lane each) rather than with 8 pieces per lane, which would spill
+  if (long_instance) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
+  if (!wide) return launch_group_mean_as<T, 4, 4, 4>(p, smem, stream);
+  return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
 }
 
 }  // namespace vscan
