@@ -317,13 +317,15 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
             host_in = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for k, v in dev_in.items()}
             outs = {"merged": red.merged, **{k: red.out2[k] for k in ("kept_vis", "hidden", "k", "v", "pos")}}
             host_out = {k: torch.empty(v.shape, dtype=v.dtype, pin_memory=True) for k, v in outs.items()}
-            e_steps = max(1, min(args.steps, 5))
-            red.run_host(host_in, host_out, dev_in)
+            e_steps = max(1, min(args.steps, 8))
+            dev_slots = [dev_in, sets[1 % n_sets]]
+            red.run_host_many([host_in] * 2, [host_out] * 2, dev_slots)
             stream.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
-            for _ in range(e_steps):
-                red.run_host(host_in, host_out, dev_in)
+            # every step uploads its inputs and downloads its results; uploads, passes and downloads
+            # of neighbouring steps overlap on three streams
+            red.run_host_many([host_in] * e_steps, [host_out] * e_steps, dev_slots)
             e1.record(stream)
             e1.synchronize()
             e_ms = max_over_ranks(e0.elapsed_time(e1), dist, device)

@@ -36,7 +36,7 @@ __device__ __forceinline__ void qk_softmax_role(const QkParams& p, const int h, 
   __shared__ SelectScratch sc;
   __shared__ int is_last;
   constexpr int E = Vec16<T>::kElems;
-  constexpr int R = 4;   // key rows in flight per 8-lane group
+  constexpr int R = VPS > 0 && VPS <= 2 ? 8 : 4;   // key rows in flight per 8-lane group
   if (h == 0 && b == 0 && threadIdx.x == 0 && p.status) *p.status = 0u;
   const int g = static_cast<int>((static_cast<long long>(h) * p.kv_heads) / p.q_heads);
   const T* qh = static_cast<const T*>(p.q) + (static_cast<size_t>(b) * p.q_heads + h) * p.head_dim;

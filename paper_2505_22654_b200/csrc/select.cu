@@ -69,8 +69,19 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
     const T* al = static_cast<const T*>(p.attn_local) + inst;
     for (int i = threadIdx.x; i < p.n; i += blockDim.x) {
       const bool same = p.attn_local == p.attn_global;
-      const float g = head_mean_of(ag + i, p.heads, p.row_len);
-      const float l = same ? g : head_mean_of(al + i, p.heads, p.row_len);
+      float g, l;
+      if (!same && p.heads == 16) {   // the common head count: all 32 loads of the token in flight at once
+        T a[16], c[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { a[u] = ag[i + static_cast<size_t>(u) * p.row_len]; c[u] = al[i + static_cast<size_t>(u) * p.row_len]; }
+        g = 0.f; l = 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { g += to_float(a[u]); l += to_float(c[u]); }
+        g /= 16.f; l /= 16.f;
+      } else {
+        g = head_mean_of(ag + i, p.heads, p.row_len);
+        l = same ? g : head_mean_of(al + i, p.heads, p.row_len);
+      }
       if (p.scores_global_out) p.scores_global_out[static_cast<size_t>(b) * p.n + i] = g;
       if (p.scores_local_out) p.scores_local_out[static_cast<size_t>(b) * p.n + i] = l;
       keys_g[i] = float_to_key(g);

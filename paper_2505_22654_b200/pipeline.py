@@ -98,3 +98,43 @@ class VScanReducer:
         for name in ("kept_vis", "hidden", "k", "v", "pos"):
             host_out[name].copy_(self.out2[name], non_blocking=True)
         return host_out
+
+    def run_host_many(self, host_ins, host_outs, dev_sets):
+        """A stream of batches from pinned host memory: the upload of batch i+1 and the download of
+        batch i-1 overlap the pass over batch i (three streams, `dev_sets` >= 2 device input sets used
+        in turn; outputs are single-buffered, so a pass waits for the previous download).  Everything
+        is enqueued asynchronously; the caller synchronises the current stream, which ends up ordered
+        after the last download."""
+        cur = torch.cuda.current_stream()
+        if not hasattr(self, "_s_in"):
+            self._s_in, self._s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        n_slots = len(dev_sets)
+        ev_in = [torch.cuda.Event() for _ in range(n_slots)]
+        ev_done = [None] * n_slots          # pass that last used the slot
+        ev_out = None                       # last download
+        self._s_in.wait_stream(cur)
+        self._s_out.wait_stream(cur)
+        for i, (hin, hout) in enumerate(zip(host_ins, host_outs)):
+            slot = i % n_slots
+            with torch.cuda.stream(self._s_in):
+                if ev_done[slot] is not None:
+                    self._s_in.wait_event(ev_done[slot])
+                for name, t in hin.items():
+                    dev_sets[slot][name].copy_(t, non_blocking=True)
+                ev_in[slot].record(self._s_in)
+            cur.wait_event(ev_in[slot])
+            if ev_out is not None:
+                cur.wait_event(ev_out)
+            self.run(**dev_sets[slot])
+            ev_done[slot] = torch.cuda.Event()
+            ev_done[slot].record(cur)
+            with torch.cuda.stream(self._s_out):
+                self._s_out.wait_event(ev_done[slot])
+                hout["merged"].copy_(self.merged, non_blocking=True)
+                for name in ("kept_vis", "hidden", "k", "v", "pos"):
+                    hout[name].copy_(self.out2[name], non_blocking=True)
+                ev_out = torch.cuda.Event()
+                ev_out.record(self._s_out)
+        if ev_out is not None:
+            cur.wait_event(ev_out)
+        return host_outs

@@ -105,3 +105,29 @@ def test_config4_sweep_batches(batch, retention):
     g = min(batch, 4)
     run_and_check(cfg, gen_instances=g * cfg.C, gen_batch=g,
                   sample=lambda n: sorted(set(np.linspace(0, n - 1, 9).astype(int).tolist())))
+
+
+def test_host_stream_of_batches_matches_device_runs():
+    """run_host_many overlaps uploads, passes and downloads of neighbouring batches; every batch's
+    results must equal those of a plain device-resident run on the same inputs."""
+    cfg = CONFIGS[2].with_(name="host_stream", B=3, C=2, k2=64)
+    red = vs.VScanReducer.from_config(cfg)
+    batches = []
+    for seed in range(4):
+        s1, s2 = stage1_case(cfg, seed=seed, planted=False), stage2_case(cfg, seed=seed, planted=False)
+        batches.append({"attn_g": dev(s1["attn_g"], cfg.dtype), "attn_l": dev(s1["attn_l"], cfg.dtype),
+                        "x": dev(s1["x"], cfg.dtype), "q_last": dev(s2["q_last"], cfg.dtype), "k": dev(s2["k"], cfg.dtype),
+                        "v": dev(s2["v"], cfg.dtype), "hidden": dev(s2["hidden"], cfg.dtype), "pos_ids": dev(s2["pos_ids"])})
+    expect = []
+    for d in batches:
+        red.run(**d)
+        torch.cuda.synchronize()
+        expect.append({"merged": red.merged.cpu().clone(), **{k: red.out2[k].cpu().clone() for k in ("kept_vis", "hidden", "k", "v", "pos")}})
+    host_ins = [{k: v.cpu().pin_memory() for k, v in d.items()} for d in batches]
+    host_outs = [{k: torch.empty_like(v).pin_memory() for k, v in e.items()} for e in expect]
+    slots = [{k: torch.empty_like(v) for k, v in batches[0].items()} for _ in range(2)]
+    red.run_host_many(host_ins, host_outs, slots)
+    torch.cuda.synchronize()
+    for got, ref in zip(host_outs, expect):
+        for name in ref:
+            assert torch.equal(got[name], ref[name]), name
