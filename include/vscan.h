@@ -60,8 +60,13 @@ typedef enum {
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
   VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group means in a
                              second kernel */
-  VSCAN_MERGE_FUSED = 3   /* norms, tcgen05 similarity + arg-max and group means in one kernel, one cluster of
+  VSCAN_MERGE_FUSED = 3,  /* norms, tcgen05 similarity + arg-max and group means in one kernel, one cluster of
                              CTAs per instance (bf16, n_kept <= 256, n_tokens <= 8192) */
+  VSCAN_MERGE_INTERLEAVED = 4 /* the TENSOR path's two steps in one launch: the CTA that has assigned a tile of
+                             one instance goes on to sum groups of an instance a few places earlier in the
+                             batch, whose features are still in L2 (bf16, n_kept <= 192, n_tokens <= 768
+                             and small enough for one 128-byte column slice of an instance to fit the
+                             CTA's shared memory) */
 } vscan_merge_path;
 
 /* ---------------------------------------------------------------------------------------------

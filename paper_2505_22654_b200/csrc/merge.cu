@@ -4,6 +4,7 @@
 //                           row of the similarity matrix and cannot change the arg-max)
 //   group_mean_kernel      members of every slot in ascending token order, fp32 sum, one rounding
 #include "merge.cuh"
+#include "merge_mean.cuh"
 
 namespace vscan {
 
@@ -151,110 +152,10 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 // dynamic shared memory: list[n_tokens] of (local slot << 24 | token), then assign[n_tokens]
 template <typename T, int VPL, int R, int kSlotsPerCta>
 __global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergeParams p) {
-  constexpr int kMeanThreads = kSlotsPerCta * 32;
-  constexpr int E = Vec16<T>::kElems;
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
-  const int b = blockIdx.y, s0 = blockIdx.x * kSlotsPerCta;
-  // all assignments of the instance -> shared memory (second half of the buffer) in one round of
-  // independent, coalesced loads; the two ordered passes below then run out of shared memory
-  int32_t* assign = reinterpret_cast<int32_t*>(list + p.n_tokens);
   grid_dependency_wait();   // the assignments come from the kernel before this one
-  {
-    const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
-    for (int i0 = threadIdx.x; i0 < p.n_tokens; i0 += kMeanThreads * 8) {
-      int32_t v[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
-#pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; if (i < p.n_tokens) assign[i] = v[u]; }
-    }
-  }
-  __syncthreads();
-
-  // contiguous run of tokens per thread; an odd run length keeps the threads of a warp on different banks
-  const int per = ((p.n_tokens + blockDim.x - 1) / blockDim.x) | 1;
-  const int lo = min(p.n_tokens, static_cast<int>(threadIdx.x) * per), hi = min(p.n_tokens, lo + per);
-  int mine = 0;
-  for (int i = lo; i < hi; ++i) {
-    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
-    mine += rel < static_cast<unsigned>(kSlotsPerCta);
-  }
-  int n_list;
-  int pos = block_exclusive_scan(mine, warp_sums, n_list);
-  for (int i = lo; i < hi; ++i) {
-    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
-    if (rel < static_cast<unsigned>(kSlotsPerCta)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
-  }
-  __syncthreads();
-
-  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, s = s0 + w;
-  if (s >= p.n_kept) return;
-  const int vecs = p.dim / E;
-  const T* xb = static_cast<const T*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
-  T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
-
-  for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
-    float acc[VPL][E];
-#pragma unroll
-    for (int i = 0; i < VPL; ++i)
-#pragma unroll
-      for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
-    int count = 0;
-    for (int c = 0; c < n_list; c += 32) {
-      const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
-      unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(w));
-      count += __popc(mask);
-      while (mask) {
-        int tok[R];
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          tok[r] = -1;
-          if (mask) {
-            const int l = __ffs(mask) - 1;
-            mask &= mask - 1;
-            tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
-          }
-        }
-        uint4 raw[R][VPL];
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
-#pragma unroll
-          for (int i = 0; i < VPL; ++i) {
-            const int v = v0 + lane + 32 * i;
-            if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
-          }
-        }
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          if (tok[r] < 0) continue;
-#pragma unroll
-          for (int i = 0; i < VPL; ++i) {
-            const int v = v0 + lane + 32 * i;
-            if (v < vecs) {
-              float f[E];
-              Vec16<T>::unpack(raw[r][i], f);
-#pragma unroll
-              for (int e = 0; e < E; ++e) acc[i][e] += f[e];
-            }
-          }
-        }
-      }
-    }
-    const float inv = 1.f / static_cast<float>(max(count, 1));
-#pragma unroll
-    for (int i = 0; i < VPL; ++i) {
-      const int v = v0 + lane + 32 * i;
-      if (v < vecs) {
-        float f[E];
-#pragma unroll
-        for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
-        st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
-      }
-    }
-    if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
-  }
+  group_mean_body<T, VPL, R, kSlotsPerCta>(p, blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums);
 }
 
 template <typename T, int VPL, int R, int SLOTS>
@@ -275,7 +176,7 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   // 512-thread CTAs have 128 registers per thread: wide rows are then summed in two column passes
   // (4 pieces per lane each) rather than with 8 pieces per lane, which would spill
   if (long_instance) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
-  if (!wide) return launch_group_mean_as<T, 4, 4, 4>(p, smem, stream);
+  if (!wide) return launch_group_mean_as<T, 2, 4, 4>(p, smem, stream);   // two column passes, 56 registers: more CTAs per SM
   return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
 }
 
@@ -287,7 +188,7 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
   if (!d || !d->x || !d->kept_idx || !d->merged) return VSCAN_ERR_INVALID_ARG;
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
   if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR &&
-      d->path != VSCAN_MERGE_FUSED)
+      d->path != VSCAN_MERGE_FUSED && d->path != VSCAN_MERGE_INTERLEAVED)
     return VSCAN_ERR_INVALID_ARG;
   if (d->instances < 0 || d->n_tokens <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + d->n_tokens ||
       d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
@@ -365,6 +266,17 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
       if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_FUSED) return st;
       p.assign = d->assign ? d->assign : ws_assign;
     } else if (d->path == VSCAN_MERGE_FUSED) {
+      return VSCAN_ERR_UNSUPPORTED;
+    }
+  }
+
+  // assignment and group sums in one launch (measured slower than the two kernels below at every batch size tried:
+  // on request only)
+  if (d->path == VSCAN_MERGE_INTERLEAVED) {
+    if (merge_interleaved_supported(d->dtype, p)) {
+      st = launch_merge_interleaved(p, stream);
+      if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_INTERLEAVED) return st;
+    } else if (d->path == VSCAN_MERGE_INTERLEAVED) {
       return VSCAN_ERR_UNSUPPORTED;
     }
   }

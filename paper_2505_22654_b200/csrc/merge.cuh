@@ -26,6 +26,11 @@ vscan_status launch_assign_simt(int dtype, const MergeParams& p, cudaStream_t st
 // cannot take.
 vscan_status launch_assign_tensor(const MergeParams& p, cudaStream_t stream);
 bool assign_tensor_supported(int dtype, const MergeParams& p);
+// Tensor-core assignment and group means in one launch (bf16, kept sets small enough for two or three
+// CTAs per SM): the mean CTAs of an instance follow its assignment CTAs in block order and re-read the
+// features from L2.  Clears the status word and uses the inv_norm region of the workspace for counters.
+vscan_status launch_merge_interleaved(const MergeParams& p, cudaStream_t stream);
+bool merge_interleaved_supported(int dtype, const MergeParams& p);
 // Norms, assignment and group means in one kernel (bf16, at most 256 kept tokens and 8192 tokens per
 // instance).  Writes merged / assign / counts directly; needs no inv_norm or assign scratch.
 vscan_status launch_merge_fused(const MergeParams& p, cudaStream_t stream);

@@ -11,6 +11,8 @@
 // The similarity matrix never leaves the SM.  Every mbarrier wait is bounded: on expiry the CTA
 // records VSCAN_ERR_TIMEOUT in the status word, lets copies in flight land, frees its tensor memory
 // and returns.
+#include <cstdlib>
+
 #include "merge.cuh"
 #include "tc_common.cuh"
 
@@ -39,7 +41,6 @@ struct Shared {
   uint32_t tmem_base;
   int abort_flag;
   int best_slot[kTileM];
-  float inv_norm[2][kMaxN];
 };
 
 // Copies the kept rows of every instance into a contiguous [instance][slot][dim] buffer (slots past
@@ -60,18 +61,22 @@ __global__ void __launch_bounds__(256) pack_kept_kernel(MergeParams m, int rows_
   }
 }
 
-// dynamic shared memory (1024-byte aligned): stages x [A tile 128x64 bf16 | B tile n_pad x 64 bf16]
-__global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_constant__ CUtensorMap map_a,
-                                                                 const __grid_constant__ CUtensorMap map_b, Params p) {
-  extern __shared__ unsigned char smem_dyn[];
-  __shared__ Shared sh;
+// The whole life of one assignment CTA: tile of 128 tokens starting at token t0 of instance b.
+// smem_dyn: up to 1023 bytes of alignment slack | stages x [A tile 128x64 bf16 | B tile n_pad x 64 bf16] |
+// inv_norm[1 or 2][n_pad] floats (kept in dynamic memory so that three CTAs fit in one SM's 228 KB).
+// `done` (optional): counter of the instance, incremented once the assignments of the tile are visible
+// device-wide (not incremented when a wait of this CTA ran out).
+__device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const CUtensorMap* map_b_ptr, const Params& p,
+                                            Shared& sh, unsigned char* smem_dyn, int b, int t0, int* done) {
+  const CUtensorMap& map_a = *map_a_ptr;
+  const CUtensorMap& map_b = *map_b_ptr;
   // the swizzle pattern is a function of the shared-memory address: stage bases sit on 1024 bytes
   unsigned char* tiles = smem_dyn + ((1024u - (static_cast<uint32_t>(__cvta_generic_to_shared(smem_dyn)) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int b = blockIdx.y, t0 = blockIdx.x * kTileM;
   const MergeParams& m = p.m;
   volatile int* abort_flag = &sh.abort_flag;
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  float* inv_norm = reinterpret_cast<float*>(tiles + p.stages * stage_bytes);   // [accumulator][n_pad]
   const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
 
   if (threadIdx.x == 0) {
@@ -86,7 +91,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (m.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
+  if (m.clear_status && b == 0 && t0 == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -204,7 +209,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         const int r = ptid + 128 * u;
-        if (r < p.n_pad) sh.inv_norm[acc][r] = (n0 + r < m.n_kept) ? 1.f / fmaxf(sqrtf(ss[u]), 1e-12f) : 0.f;
+        if (r < p.n_pad) inv_norm[acc * p.n_pad + r] = (n0 + r < m.n_kept) ? 1.f / fmaxf(sqrtf(ss[u]), 1e-12f) : 0.f;
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
@@ -224,7 +229,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
         for (int j = 0; j < 32; ++j) {
           const int s_idx = n0 + c0 + j;
           if (c0 + j < p.n_pad && s_idx < m.n_kept) {
-            const float val = __uint_as_float(v[j]) * sh.inv_norm[acc][c0 + j];
+            const float val = __uint_as_float(v[j]) * inv_norm[acc * p.n_pad + c0 + j];
             if (val > best_val) { best_val = val; best_idx = s_idx; }
           }
         }
@@ -242,6 +247,11 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (ok && t0 + ptid < m.n_tokens) m.assign[static_cast<size_t>(b) * m.n_tokens + t0 + ptid] = sh.best_slot[ptid];
+    if (done) {   // publish: the 128 stores above first, then one increment
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ptid == 0 && ok && !*abort_flag) atomicAdd(done, 1);
+    }
   }
 
   // ------------------------------------------------------------ teardown
@@ -257,6 +267,206 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(p.tmem_cols) : "memory");
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_constant__ CUtensorMap map_a,
+                                                                 const __grid_constant__ CUtensorMap map_b, Params p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ Shared sh;
+  assign_tile(&map_a, &map_b, p, sh, smem_dyn, blockIdx.y, blockIdx.x * kTileM, nullptr);
+}
+
+// Assignment and group means in ONE launch, so that the second pass over the features (the sums of
+// Eq. 4) reads them from L2 while they are still there.  The CTA that has assigned tile t of instance i
+// goes on to sum groups of instance i - lag: the column slices t, t + tiles, ... of it.  The hardware
+// hands out blocks in index order, so the tiles of instance i - lag were started lag * tiles blocks
+// earlier and have normally finished by then; the CTA still checks the instance's counter of finished
+// tiles and spins (bounded; on expiry VSCAN_ERR_TIMEOUT) until it is complete.  lag * tiles extra
+// CTAs at the end of the grid take the sums of the last `lag` instances.  Nothing waits on a block
+// with a higher index, and no CTA exists only to wait.
+struct Interleave {
+  int* done;        // [instances] finished assignment tiles, zero at launch
+  int tiles;        // assignment CTAs per instance
+  int slices;       // slices of kSliceCols feature columns
+  int x_boxes;      // tile loads (kBoxRows rows x kSliceCols columns) that cover the tokens of an instance
+  int lag;          // instances between an assignment and its sums, 1 <= lag <= instances
+};
+constexpr uint32_t kDoneSpinLimit = 1u << 22;    // polls of ~100 ns
+constexpr int kSliceCols = 64;                   // feature columns of one slice (128 bytes per row)
+constexpr int kBoxRows = 192;                    // token rows per tile load of a slice
+constexpr int kMaxBoxes = 4;
+constexpr int kMaxMeanKept = kThreads;           // kept slots the shared tables hold (one thread per slot in the sort)
+constexpr int kWarps = kThreads / 32;
+
+struct MeanShared {
+  uint64_t full;                       // the current column slice has landed
+  uint32_t tmem_base;
+  int ready;                           // assignments of the instance complete (0: the wait ran out)
+  int warp_sums[33];
+  uint16_t begin[kMaxMeanKept + 2];    // first list position of each slot; begin[n_kept] = listed tokens
+};
+
+// Sums of the slices `first`, `first + il.tiles`, ... of instance b (a slice = kSliceCols feature columns).
+//   1. wait for the instance's assignments; 2. a stable counting sort of its tokens by slot (every slot's
+//   members in ascending token order): a bit mask per (slot, 32-token chunk) filled with shared-memory
+//   atomics, prefix sums over chunks and slots, then every mask word writes out its tokens; 3. per slice:
+//   the 128-byte column slice of all tokens comes in by a few tile loads, then groups of 8 lanes (16
+//   bytes each) walk the member lists, one slot per group at a time, adding in list order in fp32, one
+//   rounding.  Same order of additions as group_mean_body, hence the same bits.
+// smem_dyn: the slice (n_tokens rounded up to boxes x 128 bytes; the sort's scratch before the first
+// slice is fetched) followed by the member list (n_tokens x 2 bytes).
+__device__ __forceinline__ void mean_share(const CUtensorMap* map_x, const MergeParams& m, const Interleave& il,
+                                           MeanShared& ms, unsigned char* smem_dyn, int b, int first) {
+  constexpr int kRowBytes = kSliceCols * 2, kLanesPerRow = kRowBytes / 16;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned char* tiles = smem_dyn + ((128u - (smem_u32(smem_dyn) & 127u)) & 127u);
+  const uint32_t slice_bytes = static_cast<uint32_t>(il.x_boxes) * kBoxRows * kRowBytes;
+  uint16_t* list = reinterpret_cast<uint16_t*>(tiles + slice_bytes);
+  const int chunks = (m.n_tokens + 31) / 32;
+  uint32_t* bits = reinterpret_cast<uint32_t*>(tiles);                       // [n_kept][chunks] (scratch)
+  uint16_t* offs = reinterpret_cast<uint16_t*>(bits + m.n_kept * chunks);    // [n_kept][chunks] (scratch)
+  if (threadIdx.x == 0) {
+    mbar_init(&ms.full, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const volatile int* flag = il.done + b;
+    uint32_t spins = 0;
+    while (*flag < il.tiles && spins < kDoneSpinLimit) { __nanosleep(100); ++spins; }
+    ms.ready = *flag >= il.tiles;
+    if (!ms.ready) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+    __threadfence();
+  }
+  for (int i = threadIdx.x; i < m.n_kept * chunks; i += kThreads) bits[i] = 0u;
+  __syncthreads();
+  if (!ms.ready) return;
+
+  // ---- sort
+  const int32_t* ag = m.assign + static_cast<size_t>(b) * m.n_tokens;
+  for (int c = warp; c < chunks; c += kWarps) {
+    const int t = c * 32 + lane;
+    if (t < m.n_tokens) {
+      const int v = __ldcg(ag + t);
+      if (v >= 0 && v < m.n_kept) atomicOr(&bits[v * chunks + c], 1u << lane);
+    }
+  }
+  __syncthreads();
+  int total = 0;
+  if (threadIdx.x < m.n_kept) {
+    for (int c = 0; c < chunks; ++c) {
+      offs[threadIdx.x * chunks + c] = static_cast<uint16_t>(total);
+      total += __popc(bits[threadIdx.x * chunks + c]);
+    }
+  }
+  int listed;
+  const int start = block_exclusive_scan(total, ms.warp_sums, listed);   // contains the barriers
+  if (threadIdx.x < m.n_kept) ms.begin[threadIdx.x] = static_cast<uint16_t>(start);
+  if (threadIdx.x == 0) ms.begin[m.n_kept] = static_cast<uint16_t>(listed);
+  __syncthreads();
+  for (int i = threadIdx.x; i < m.n_kept * chunks; i += kThreads) {
+    const int sl = i / chunks, c = i - sl * chunks;
+    uint32_t word = bits[i];
+    int pos = ms.begin[sl] + offs[i];
+    while (word) {
+      const int bit = __ffs(word) - 1;
+      word &= word - 1;
+      list[pos++] = static_cast<uint16_t>(c * 32 + bit);
+    }
+  }
+  __syncthreads();   // the list is complete and the scratch is free
+
+  // ---- slices
+  volatile int local_abort = 0;
+  const int group = threadIdx.x / kLanesPerRow, piece = threadIdx.x % kLanesPerRow;
+  int round = 0;
+  for (int slice = first; slice < il.slices; slice += il.tiles, ++round) {
+    if (threadIdx.x == 0) {
+      mbar_arrive_expect_tx(&ms.full, slice_bytes);
+      for (int i = 0; i < il.x_boxes; ++i)
+        tma_load_3d(tiles + static_cast<size_t>(i) * kBoxRows * kRowBytes, map_x, &ms.full, slice * kSliceCols,
+                    m.cls_offset + i * kBoxRows, b);
+    }
+    // every thread waits itself: the slice was written by the copy engine
+    const bool landed = mbar_wait(&ms.full, round & 1, &local_abort);
+    if (!landed) {   // (all threads of the CTA wait on the same phase: they give up together)
+      if (threadIdx.x == 0) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+      for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let the copies land before the memory is released
+      return;
+    }
+    const unsigned char* rows = tiles + piece * 16;
+    const int col = slice * kSliceCols + piece * 8;
+    for (int sl = group; sl < m.n_kept; sl += kThreads / kLanesPerRow) {
+      const int k0 = ms.begin[sl], k1 = ms.begin[sl + 1];
+      float acc[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+      for (int k = k0; k < k1; k += 4) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (k + u < k1) v[u] = *reinterpret_cast<const uint4*>(rows + static_cast<uint32_t>(list[k + u]) * kRowBytes);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (k + u < k1) {
+            float f[8];
+            Vec16<__nv_bfloat16>::unpack(v[u], f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[e] += f[e];
+          }
+        }
+      }
+      const int count = k1 - k0;
+      const float inv = 1.f / static_cast<float>(max(count, 1));
+      if (col < m.dim) {
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) f[e] = acc[e] * inv;
+        st_16(static_cast<__nv_bfloat16*>(m.merged) + (static_cast<size_t>(b) * m.n_kept + sl) * m.dim + col,
+              Vec16<__nv_bfloat16>::pack(f));
+      }
+      if (slice == 0 && piece == 0 && m.counts) m.counts[static_cast<size_t>(b) * m.n_kept + sl] = count;
+    }
+    __syncthreads();   // every thread has read the slice: the next one may overwrite it
+  }
+}
+
+template <int kMinCtas>
+__global__ void __launch_bounds__(kThreads, kMinCtas)
+merge_interleaved_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                         const __grid_constant__ CUtensorMap map_x, Params p, Interleave il) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ Shared sh;
+  __shared__ MeanShared ms;
+  const int n_assign = p.m.instances * il.tiles, bid = blockIdx.x;
+  int mean_b, part;
+  if (bid < n_assign) {
+    const int b = bid / il.tiles;
+    part = bid - b * il.tiles;
+    assign_tile(&map_a, &map_b, p, sh, smem_dyn, b, part * kTileM, il.done + b);
+    mean_b = b - il.lag;
+    if (mean_b < 0) return;
+    __syncthreads();   // the tile's teardown is complete: shared memory changes hands
+  } else {
+    const int r = bid - n_assign;
+    mean_b = p.m.instances - il.lag + r / il.tiles;
+    part = r - (r / il.tiles) * il.tiles;
+    // A CTA of a kernel that uses tensor memory keeps the right to allocate it until it gives that right
+    // up, and the SM starts no further CTA of the kernel beside it meanwhile: take the smallest
+    // allocation and relinquish at once, as the assignment CTAs do.
+    if (threadIdx.x < 32) {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)), "r"(32) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    grid_dependency_launch();
+    grid_dependency_wait();   // the features may come from the kernel before this one
+  }
+  mean_share(&map_x, p.m, il, ms, smem_dyn, mean_b, part);
+  if (bid >= n_assign) {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(ms.tmem_base), "r"(32) : "memory");
+    }
   }
 }
 
@@ -284,6 +494,12 @@ static bool plan(const MergeParams& m, Params& p) {
   return stages >= 2;
 }
 
+// dynamic shared memory of an assignment CTA: alignment slack, the stage ring, the inverse norms
+static size_t smem_bytes(const Params& p) {
+  return 1024 + static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) +
+         static_cast<size_t>(p.n_chunks > 1 ? 2 : 1) * p.n_pad * sizeof(float);
+}
+
 }  // namespace tc
 
 bool assign_tensor_supported(int dtype, const MergeParams& m) {
@@ -293,12 +509,11 @@ bool assign_tensor_supported(int dtype, const MergeParams& m) {
   return tc::plan(m, p) && tc::encode_fn() != nullptr;
 }
 
-vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
-  tc::Params p;
-  if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
+// Tensor maps of a launch: the token tiles (3-D [instance][row][dim]) and the kept rows (the same memory
+// as a 2-D [all rows][dim] tensor for row gathers, or the packed copy for large kept sets).
+static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUtensorMap& map, CUtensorMap& map_b) {
   tc::EncodeTiledFn encode = tc::encode_fn();
   if (!encode) return VSCAN_ERR_UNSUPPORTED;
-  CUtensorMap map;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(m.metric_dim), static_cast<cuuint64_t>(m.row_len),
                               static_cast<cuuint64_t>(m.instances)};
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(m.metric_dim) * 2,
@@ -309,8 +524,6 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
                       elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
-  // kept rows: the same memory as a 2-D [all rows][dim] tensor, fetched four rows at a time
-  CUtensorMap map_b;
   const cuuint64_t dims_b[2] = {static_cast<cuuint64_t>(m.metric_dim),
                                 static_cast<cuuint64_t>(m.row_len) * static_cast<cuuint64_t>(m.instances)};
   const cuuint64_t strides_b[1] = {static_cast<cuuint64_t>(m.metric_dim) * 2};
@@ -329,16 +542,103 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   }
-  if (r != CUDA_SUCCESS) return VSCAN_ERR_UNSUPPORTED;
+  return r == CUDA_SUCCESS ? VSCAN_OK : VSCAN_ERR_UNSUPPORTED;
+}
+
+vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
+  tc::Params p;
+  if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
+  CUtensorMap map, map_b;
+  vscan_status st = encode_maps(m, p, map, map_b);
+  if (st != VSCAN_OK) return st;
   if (p.b_packed) {
     dim3 pgrid((static_cast<unsigned>(p.n_chunks) * p.n_pad + 7) / 8, m.instances);
     VSCAN_LAUNCH("pack_kept", stream, tc::pack_kept_kernel<<<pgrid, 256, 0, stream>>>(m, p.n_chunks * p.n_pad));
   }
-  const size_t smem = static_cast<size_t>(p.stages) * (p.a_stage_bytes + p.b_stage_bytes) + 1024;
+  const size_t smem = tc::smem_bytes(p);
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
   dim3 grid((m.n_tokens + tc::kTileM - 1) / tc::kTileM, m.instances);
   VSCAN_LAUNCH("assign_tensor", stream,
                (void)launch_dependent(tc::assign_tensor_kernel, grid, dim3(tc::kThreads), smem, stream, map, map_b, p));
+  return VSCAN_OK;
+}
+
+// ---- assignment + group means in one launch
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+    else return 148;
+  }
+  return n;
+}
+
+static bool plan_interleaved(const MergeParams& m, tc::Params& p, tc::Interleave& il, int& ctas_per_sm, size_t& smem) {
+  if (!tc::plan(m, p) || p.n_chunks != 1 || p.b_packed) return false;
+  const int stage = p.a_stage_bytes + p.b_stage_bytes;
+  ctas_per_sm = (73 * 1024) / stage >= 3 ? 3 : ((110 * 1024) / stage >= 3 ? 2 : 1);
+  smem = tc::smem_bytes(p);
+  // the sums: the column slice of every token (whole tile loads) + the member list
+  il.x_boxes = (m.n_tokens + tc::kBoxRows - 1) / tc::kBoxRows;
+  if (il.x_boxes > tc::kMaxBoxes || m.n_kept > tc::kMaxMeanKept) return false;
+  const size_t slice_bytes = static_cast<size_t>(il.x_boxes) * tc::kBoxRows * tc::kSliceCols * 2;
+  if (128 + slice_bytes + static_cast<size_t>(m.n_tokens) * 2 > smem) return false;
+  if (static_cast<size_t>(m.n_kept) * ((m.n_tokens + 31) / 32) * 6 > slice_bytes) return false;   // the sort's scratch
+  if ((reinterpret_cast<uintptr_t>(m.x) & 15u) != 0 || m.dim % 8 != 0) return false;
+  il.done = reinterpret_cast<int*>(m.inv_norm);   // the tensor path takes the norms itself: the region is free
+  il.tiles = (m.n_tokens + tc::kTileM - 1) / tc::kTileM;
+  il.slices = (m.dim + tc::kSliceCols - 1) / tc::kSliceCols;
+  // far enough back that the instance's tiles have finished, near enough that its features are still in L2
+  int lag = 16;
+  if (const char* e = getenv("VSCAN_MERGE_LAG")) lag = atoi(e) > 0 ? atoi(e) : lag;
+  il.lag = lag < m.instances ? lag : m.instances;
+  if ((static_cast<long long>(m.instances) + il.lag) * il.tiles > 0x7fffffffLL) return false;
+  return true;
+}
+
+bool merge_interleaved_supported(int dtype, const MergeParams& m) {
+  if (!assign_tensor_supported(dtype, m)) return false;
+  tc::Params p; tc::Interleave il; int c; size_t smem;
+  return plan_interleaved(m, p, il, c, smem);
+}
+
+vscan_status launch_merge_interleaved(const MergeParams& m_in, cudaStream_t stream) {
+  MergeParams m = m_in;
+  m.clear_status = 0;   // the memset below clears the status word together with the counters
+  tc::Params p; tc::Interleave il; int ctas_per_sm; size_t smem;
+  if (!plan_interleaved(m, p, il, ctas_per_sm, smem)) return VSCAN_ERR_UNSUPPORTED;
+  CUtensorMap map, map_b, map_x;
+  vscan_status st = encode_maps(m, p, map, map_b);
+  if (st != VSCAN_OK) return st;
+  {   // column slices of the features for the sums: [instance][row][dim], box = kSliceCols columns x kBoxRows rows
+    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(m.dim), static_cast<cuuint64_t>(m.row_len),
+                                static_cast<cuuint64_t>(m.instances)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(m.dim) * 2, static_cast<cuuint64_t>(m.row_len) * m.dim * 2};
+    const cuuint32_t box[3] = {tc::kSliceCols, tc::kBoxRows, 1};
+    const cuuint32_t elem[3] = {1, 1, 1};
+    if (tc::encode_fn()(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(m.x), dims, strides, box, elem,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return VSCAN_ERR_UNSUPPORTED;
+  }
+  // status word (first 256 bytes of the workspace) and the counters right behind it
+  if (reinterpret_cast<char*>(il.done) != reinterpret_cast<char*>(m.status) + kStatusBytes) return VSCAN_ERR_WORKSPACE;
+  VSCAN_CUDA_TRY(cudaMemsetAsync(m.status, 0, kStatusBytes + static_cast<size_t>(m.instances) * sizeof(int), stream));
+  const unsigned blocks = static_cast<unsigned>(m.instances + il.lag) * il.tiles;
+  if (ctas_per_sm == 3) {
+    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<3>, smem));
+    VSCAN_LAUNCH("merge_interleaved", stream,
+                 (void)launch_dependent(tc::merge_interleaved_kernel<3>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
+  } else if (ctas_per_sm == 2) {
+    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<2>, smem));
+    VSCAN_LAUNCH("merge_interleaved", stream,
+                 (void)launch_dependent(tc::merge_interleaved_kernel<2>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
+  } else {
+    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<1>, smem));
+    VSCAN_LAUNCH("merge_interleaved", stream,
+                 (void)launch_dependent(tc::merge_interleaved_kernel<1>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
+  }
   return VSCAN_OK;
 }
 

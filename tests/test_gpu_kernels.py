@@ -166,7 +166,7 @@ def test_merge_exact_ties_and_duplicates():
 
 @pytest.mark.parametrize("N,D,K1,c", [(576, 1024, 64, 1), (576, 1024, 192, 1), (300, 72, 17, 0), (130, 264, 130, 1),
                                       (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0)])
-@pytest.mark.parametrize("path", ["tensor", "fused"])
+@pytest.mark.parametrize("path", ["tensor", "fused", "interleaved"])
 def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     """The tcgen05 path on its own (path = TENSOR): tile tails, kept counts that are not multiples of
     16, more than 256 kept tokens (several accumulator rounds), feature dims that are not multiples
@@ -180,16 +180,48 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
             vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_FUSED)
         assert e.value.status == 2       # more kept tokens than one accumulator holds: not this path
         return
+    if path == "interleaved" and K1 > 192:
+        with pytest.raises(vs.VScanError) as e:
+            vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_INTERLEAVED)
+        assert e.value.status == 2       # more kept slots than the single-launch path's tables hold
+        return
     ws = vs.Workspace(8 << 20)
     merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
                                             want_counts=True, workspace=ws,
-                                            path=vs.MERGE_TENSOR if path == "tensor" else vs.MERGE_FUSED)
+                                            path={"tensor": vs.MERGE_TENSOR, "fused": vs.MERGE_FUSED,
+                                                  "interleaved": vs.MERGE_INTERLEAVED}[path])
     assert vs.vscan_check(ws) == 0
     for b in range(2):
         m, a, cn = vo.merge(x[b], c, kept[b])
         np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
         np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
         check_merged(merged[b], m, "bf16")
+
+
+@pytest.mark.parametrize("B,N,D,K1", [(150, 200, 64, 20), (97, 131, 128, 7), (40, 576, 1024, 64)])
+def test_merge_interleaved_many_instances(B, N, D, K1):
+    """More instances than the block-order distance between an instance's assignment CTAs and its mean
+    CTAs (head, steady part and tail of the block order all occur); two calls on one workspace (the
+    counters are cleared by every call); same result as the two-kernel tensor path, checked against
+    the oracle on sampled instances."""
+    rng = np.random.default_rng(B * 1000 + N)
+    x = round_to_dtype(rng.standard_normal((B, N, D)).astype(np.float32), "bf16")
+    kept = np.stack([np.sort(rng.choice(N, K1, replace=False)) for _ in range(B)]).astype(np.int32)
+    xd, kd = dev(x, "bf16"), dev(kept)
+    ws = vs.Workspace(8 << 20)
+    ref = vs.vscan_merge(xd, 0, kd, want_assign=True, want_counts=True, path=vs.MERGE_TENSOR)
+    for _ in range(2):
+        out = vs.vscan_merge(xd, 0, kd, want_assign=True, want_counts=True, workspace=ws, path=vs.MERGE_INTERLEAVED)
+        assert vs.vscan_check(ws) == 0
+        for r, o in zip(ref, out):
+            assert torch.equal(r, o)
+    for b in (0, B // 2, B - 1):
+        m, a, cn = vo.merge(x[b], 0, kept[b])
+        agree = out[1][b].cpu().numpy() == a      # unplanted inputs: near-ties may differ, the rest must not
+        assert agree.mean() > 0.98
+        if agree.all():
+            np.testing.assert_array_equal(out[2][b].cpu().numpy(), cn)
+            check_merged(out[0][b], m, "bf16")
 
 
 def test_merge_tensor_path_refuses_fp32():

@@ -50,8 +50,15 @@ def test_random_stage1(seed):
     x = round_to_dtype(rng.standard_normal((B, N + c, D)).astype(np.float32), dtype)
     plant.plant_merge(cfg, x, ref)
     paths = [vs.MERGE_AUTO, vs.MERGE_SIMT] + ([vs.MERGE_TENSOR, vs.MERGE_FUSED] if dtype == "bf16" and ref.shape[1] <= 256 else [])
+    if dtype == "bf16" and ref.shape[1] <= 128:
+        paths.append(vs.MERGE_INTERLEAVED)
     for path in paths:
-        merged, assign, counts = vs.vscan_merge(dev(x, dtype), c, kept, path=path, want_assign=True, want_counts=True)
+        try:
+            merged, assign, counts = vs.vscan_merge(dev(x, dtype), c, kept, path=path, want_assign=True, want_counts=True)
+        except vs.VScanError as e:
+            if path == vs.MERGE_INTERLEAVED and e.status == 2:   # shape outside the single-launch path
+                continue
+            raise
         for b in range(B):
             m, a, cn = vo.merge(x[b], c, ref[b])
             np.testing.assert_array_equal(assign[b].cpu().numpy(), a, err_msg=f"path {path}")
