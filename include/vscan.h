@@ -56,17 +56,17 @@ typedef enum { VSCAN_SCORE_ROW = 0, VSCAN_SCORE_QK = 1 } vscan_score_mode;
 typedef enum { VSCAN_SPAN_ONLY = 0, VSCAN_SPAN_FULL = 1 } vscan_softmax_span;
 /* Which unit runs the similarity contraction of vscan_merge. */
 typedef enum {
-  VSCAN_MERGE_AUTO = 0,   /* tensor cores for bf16 when the shape allows, else CUDA cores */
+  VSCAN_MERGE_AUTO = 0,   /* bf16: INTERLEAVED for kept sets of 129..256, else TENSOR when the shape allows, else SIMT;
+                             f32: SIMT */
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
   VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group means in a
                              second kernel */
   VSCAN_MERGE_FUSED = 3,  /* norms, tcgen05 similarity + arg-max and group means in one kernel, one cluster of
                              CTAs per instance (bf16, n_kept <= 256, n_tokens <= 8192) */
-  VSCAN_MERGE_INTERLEAVED = 4 /* the TENSOR path's two steps in one launch: the CTA that has assigned a tile of
-                             one instance goes on to sum groups of an instance a few places earlier in the
-                             batch, whose features are still in L2 (bf16, n_kept <= 192, n_tokens <= 768
-                             and small enough for one 128-byte column slice of an instance to fit the
-                             CTA's shared memory) */
+  VSCAN_MERGE_INTERLEAVED = 4 /* the TENSOR path's two steps in one persistent launch, one CTA per SM: six warps
+                             assign tile after tile (kept rows packed and their norms taken by a small
+                             kernel first), eight more warps sum the groups of every instance whose tiles are
+                             all done, reading its features from L2 (bf16, n_kept <= 256) */
 } vscan_merge_path;
 
 /* ---------------------------------------------------------------------------------------------

@@ -215,14 +215,19 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
   return VSCAN_OK;
 }
 
+// rows per instance of the packed copy of the kept rows: whole 256-row rounds for large kept sets, else
+// the kept count rounded up to the MMA's granularity of 16
+static size_t packed_rows(int n_kept) { return n_kept > 256 ? round_up(n_kept, 256) : round_up(n_kept, 16); }
+
 extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
   if (!d || d->instances <= 0 || d->n_kept <= 0 || d->n_tokens <= 0) return kStatusBytes;
   size_t bytes = kStatusBytes;
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256);    // inv_norm
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);  // assign
-  if (d->dtype == VSCAN_BF16 && d->n_kept > 256) {   // packed copy of the kept rows for the tensor path
+  if (d->dtype == VSCAN_BF16) {   // packed copy of the kept rows for the tensor paths
     const size_t md = d->metric ? d->metric_dim : d->dim;
-    bytes += round_up(static_cast<size_t>(d->instances) * round_up(d->n_kept, 256) * md * 2, 256);
+    bytes += round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * md * 2, 256);
+    bytes += round_up((static_cast<size_t>(d->instances) + 1) * sizeof(int), 256);   // counters of the persistent path
   }
   return bytes;
 }
@@ -248,10 +253,13 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   int32_t* ws_assign = reinterpret_cast<int32_t*>(
       ws + kStatusBytes + round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256));
   p.assign = d->assign ? d->assign : ws_assign;
-  p.kept_packed = (d->dtype == VSCAN_BF16 && d->n_kept > 256)
+  p.kept_packed = d->dtype == VSCAN_BF16
                       ? static_cast<void*>(reinterpret_cast<char*>(ws_assign) +
                                            round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256))
                       : nullptr;
+  p.counters = p.kept_packed ? reinterpret_cast<int*>(static_cast<char*>(p.kept_packed) +
+                                                      round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * p.metric_dim * 2, 256))
+                             : nullptr;
   p.merged = d->merged; p.counts = d->counts;
   p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
@@ -270,9 +278,9 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
     }
   }
 
-  // assignment and group sums in one launch (measured slower than the two kernels below at every batch size tried:
-  // on request only)
-  if (d->path == VSCAN_MERGE_INTERLEAVED) {
+  // assignment and group means in one persistent launch: on request, or by itself where it measured faster
+  // than the two kernels below (kept sets above 128, where those run one or two CTAs per SM)
+  if (d->path == VSCAN_MERGE_INTERLEAVED || (d->path == VSCAN_MERGE_AUTO && d->n_kept > 128)) {
     if (merge_interleaved_supported(d->dtype, p)) {
       st = launch_merge_interleaved(p, stream);
       if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_INTERLEAVED) return st;

@@ -277,196 +277,415 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
   assign_tile(&map_a, &map_b, p, sh, smem_dyn, blockIdx.y, blockIdx.x * kTileM, nullptr);
 }
 
-// Assignment and group means in ONE launch, so that the second pass over the features (the sums of
-// Eq. 4) reads them from L2 while they are still there.  The CTA that has assigned tile t of instance i
-// goes on to sum groups of instance i - lag: the column slices t, t + tiles, ... of it.  The hardware
-// hands out blocks in index order, so the tiles of instance i - lag were started lag * tiles blocks
-// earlier and have normally finished by then; the CTA still checks the instance's counter of finished
-// tiles and spins (bounded; on expiry VSCAN_ERR_TIMEOUT) until it is complete.  lag * tiles extra
-// CTAs at the end of the grid take the sums of the last `lag` instances.  Nothing waits on a block
-// with a higher index, and no CTA exists only to wait.
-struct Interleave {
-  int* done;        // [instances] finished assignment tiles, zero at launch
-  int tiles;        // assignment CTAs per instance
-  int slices;       // slices of kSliceCols feature columns
-  int x_boxes;      // tile loads (kBoxRows rows x kSliceCols columns) that cover the tokens of an instance
-  int lag;          // instances between an assignment and its sums, 1 <= lag <= instances
-};
-constexpr uint32_t kDoneSpinLimit = 1u << 22;    // polls of ~100 ns
-constexpr int kSliceCols = 64;                   // feature columns of one slice (128 bytes per row)
-constexpr int kBoxRows = 192;                    // token rows per tile load of a slice
-constexpr int kMaxBoxes = 4;
-constexpr int kMaxMeanKept = kThreads;           // kept slots the shared tables hold (one thread per slot in the sort)
-constexpr int kWarps = kThreads / 32;
+// Assignment and group means in ONE persistent launch (one CTA per SM), so that the second pass over the
+// features (the sums of Eq. 4) reads them from L2 while they are still there, the start-up cost of a CTA
+// is paid once per SM instead of once per tile, and the read-back of one tile overlaps the MMAs of the next.
+//   warps 0-5   the assignment roles of assign_tile (producer, MMA issuer, four read-back warps), looping
+//               over tiles blockIdx.x, blockIdx.x + gridDim.x, ...; two accumulators alternate between
+//               tiles; after a tile's assignments are visible device-wide the instance's counter of
+//               finished tiles goes up by one
+//   warps 6-13  the mean group: takes jobs (16 kept slots of one instance) off a global counter in
+//               order, waits (bounded spin; on expiry VSCAN_ERR_TIMEOUT) until the instance's tiles are
+//               all finished, lists the members of its slots and sums them, one warp per slot, exactly as
+//               group_mean_body does (same order of additions, same bits)
+// The assignment warps never wait for a mean group, and every CTA of the grid is resident at once (the
+// grid has at most one CTA per SM), so the waits of the mean groups end.
+constexpr int kMeanWarps = 8, kMeanThreads = kMeanWarps * 32;
+constexpr int kPersistThreads = kThreads + kMeanThreads;
+constexpr int kJobSlots = 16;                      // kept slots per mean job: two per warp
+constexpr uint32_t kDoneSpinLimit = 1u << 22;      // polls of ~100 ns
 
-struct MeanShared {
-  uint64_t full;                       // the current column slice has landed
-  uint32_t tmem_base;
-  int ready;                           // assignments of the instance complete (0: the wait ran out)
+struct Persist {
+  int* done;              // [instances] finished assignment tiles, zero at launch
+  int* job_head;          // next mean job, zero at launch
+  int tiles;              // tiles per instance
+  int total_tiles;
+  int jobs_per_instance;
+  int total_jobs;
+};
+
+struct PersistShared {
+  Shared a;
   int warp_sums[33];
-  uint16_t begin[kMaxMeanKept + 2];    // first list position of each slot; begin[n_kept] = listed tokens
+  int job, ready;
 };
 
-// Sums of the slices `first`, `first + il.tiles`, ... of instance b (a slice = kSliceCols feature columns).
-//   1. wait for the instance's assignments; 2. a stable counting sort of its tokens by slot (every slot's
-//   members in ascending token order): a bit mask per (slot, 32-token chunk) filled with shared-memory
-//   atomics, prefix sums over chunks and slots, then every mask word writes out its tokens; 3. per slice:
-//   the 128-byte column slice of all tokens comes in by a few tile loads, then groups of 8 lanes (16
-//   bytes each) walk the member lists, one slot per group at a time, adding in list order in fp32, one
-//   rounding.  Same order of additions as group_mean_body, hence the same bits.
-// smem_dyn: the slice (n_tokens rounded up to boxes x 128 bytes; the sort's scratch before the first
-// slice is fetched) followed by the member list (n_tokens x 2 bytes).
-__device__ __forceinline__ void mean_share(const CUtensorMap* map_x, const MergeParams& m, const Interleave& il,
-                                           MeanShared& ms, unsigned char* smem_dyn, int b, int first) {
-  constexpr int kRowBytes = kSliceCols * 2, kLanesPerRow = kRowBytes / 16;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  unsigned char* tiles = smem_dyn + ((128u - (smem_u32(smem_dyn) & 127u)) & 127u);
-  const uint32_t slice_bytes = static_cast<uint32_t>(il.x_boxes) * kBoxRows * kRowBytes;
-  uint16_t* list = reinterpret_cast<uint16_t*>(tiles + slice_bytes);
-  const int chunks = (m.n_tokens + 31) / 32;
-  uint32_t* bits = reinterpret_cast<uint32_t*>(tiles);                       // [n_kept][chunks] (scratch)
-  uint16_t* offs = reinterpret_cast<uint16_t*>(bits + m.n_kept * chunks);    // [n_kept][chunks] (scratch)
-  if (threadIdx.x == 0) {
-    mbar_init(&ms.full, 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    const volatile int* flag = il.done + b;
-    uint32_t spins = 0;
-    while (*flag < il.tiles && spins < kDoneSpinLimit) { __nanosleep(100); ++spins; }
-    ms.ready = *flag >= il.tiles;
-    if (!ms.ready) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
-    __threadfence();
-  }
-  for (int i = threadIdx.x; i < m.n_kept * chunks; i += kThreads) bits[i] = 0u;
-  __syncthreads();
-  if (!ms.ready) return;
+__device__ __forceinline__ void mean_group_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kMeanThreads) : "memory"); }
 
-  // ---- sort
-  const int32_t* ag = m.assign + static_cast<size_t>(b) * m.n_tokens;
-  for (int c = warp; c < chunks; c += kWarps) {
-    const int t = c * 32 + lane;
-    if (t < m.n_tokens) {
-      const int v = __ldcg(ag + t);
-      if (v >= 0 && v < m.n_kept) atomicOr(&bits[v * chunks + c], 1u << lane);
-    }
+// Exclusive prefix sum over the 256 threads of the mean group (named barrier 2).
+__device__ __forceinline__ int mean_group_scan(int v, int* warp_sums, int& total, int gwarp, int lane) {
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
   }
-  __syncthreads();
-  int total = 0;
-  if (threadIdx.x < m.n_kept) {
-    for (int c = 0; c < chunks; ++c) {
-      offs[threadIdx.x * chunks + c] = static_cast<uint16_t>(total);
-      total += __popc(bits[threadIdx.x * chunks + c]);
+  mean_group_sync();   // protect warp_sums from a previous use
+  if (lane == 31) warp_sums[gwarp] = incl;
+  mean_group_sync();
+  if (gwarp == 0) {
+    const int w = lane < kMeanWarps ? warp_sums[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
     }
+    if (lane < kMeanWarps) warp_sums[lane] = wi - w;
+    if (lane == 31) warp_sums[32] = wi;
   }
-  int listed;
-  const int start = block_exclusive_scan(total, ms.warp_sums, listed);   // contains the barriers
-  if (threadIdx.x < m.n_kept) ms.begin[threadIdx.x] = static_cast<uint16_t>(start);
-  if (threadIdx.x == 0) ms.begin[m.n_kept] = static_cast<uint16_t>(listed);
-  __syncthreads();
-  for (int i = threadIdx.x; i < m.n_kept * chunks; i += kThreads) {
-    const int sl = i / chunks, c = i - sl * chunks;
-    uint32_t word = bits[i];
-    int pos = ms.begin[sl] + offs[i];
-    while (word) {
-      const int bit = __ffs(word) - 1;
-      word &= word - 1;
-      list[pos++] = static_cast<uint16_t>(c * 32 + bit);
-    }
-  }
-  __syncthreads();   // the list is complete and the scratch is free
+  mean_group_sync();
+  total = warp_sums[32];
+  return warp_sums[gwarp] + incl - v;
+}
 
-  // ---- slices
-  volatile int local_abort = 0;
-  const int group = threadIdx.x / kLanesPerRow, piece = threadIdx.x % kLanesPerRow;
-  int round = 0;
-  for (int slice = first; slice < il.slices; slice += il.tiles, ++round) {
-    if (threadIdx.x == 0) {
-      mbar_arrive_expect_tx(&ms.full, slice_bytes);
-      for (int i = 0; i < il.x_boxes; ++i)
-        tma_load_3d(tiles + static_cast<size_t>(i) * kBoxRows * kRowBytes, map_x, &ms.full, slice * kSliceCols,
-                    m.cls_offset + i * kBoxRows, b);
+// One mean job: slots s0 .. s0 + kJobSlots - 1 of instance b.  `list`: 2 * n_tokens words of shared memory.
+template <int VPL, int R>
+__device__ __forceinline__ void mean_job(const MergeParams& p, int b, int s0, uint32_t* list, int* warp_sums, int gtid) {
+  constexpr int E = 8;
+  const int gwarp = gtid >> 5, lane = gtid & 31;
+  int32_t* assign = reinterpret_cast<int32_t*>(list + p.n_tokens);
+  {
+    const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
+    for (int i0 = gtid; i0 < p.n_tokens; i0 += kMeanThreads * 4) {
+      int32_t v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int i = i0 + u * kMeanThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) { const int i = i0 + u * kMeanThreads; if (i < p.n_tokens) assign[i] = v[u]; }
     }
-    // every thread waits itself: the slice was written by the copy engine
-    const bool landed = mbar_wait(&ms.full, round & 1, &local_abort);
-    if (!landed) {   // (all threads of the CTA wait on the same phase: they give up together)
-      if (threadIdx.x == 0) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
-      for (int i = 0; i < 64; ++i) __nanosleep(2000);   // let the copies land before the memory is released
-      return;
-    }
-    const unsigned char* rows = tiles + piece * 16;
-    const int col = slice * kSliceCols + piece * 8;
-    for (int sl = group; sl < m.n_kept; sl += kThreads / kLanesPerRow) {
-      const int k0 = ms.begin[sl], k1 = ms.begin[sl + 1];
-      float acc[8];
+  }
+  mean_group_sync();
+  // contiguous run of tokens per thread; an odd run length keeps the threads of a warp on different banks
+  const int per = ((p.n_tokens + kMeanThreads - 1) / kMeanThreads) | 1;
+  const int lo = min(p.n_tokens, gtid * per), hi = min(p.n_tokens, lo + per);
+  int mine = 0;
+  for (int i = lo; i < hi; ++i) mine += static_cast<unsigned>(assign[i] - s0) < static_cast<unsigned>(kJobSlots);
+  int n_list;
+  int pos = mean_group_scan(mine, warp_sums, n_list, gwarp, lane);
+  for (int i = lo; i < hi; ++i) {
+    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
+    if (rel < static_cast<unsigned>(kJobSlots)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
+  }
+  mean_group_sync();
+
+  const int vecs = p.dim / E;
+  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
+  for (int sl = gwarp; sl < kJobSlots; sl += kMeanWarps) {
+    const int s = s0 + sl;
+    if (s >= p.n_kept) break;
+    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
+    for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
+      float acc[VPL][E];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-      for (int k = k0; k < k1; k += 4) {
-        uint4 v[4];
+      for (int i = 0; i < VPL; ++i)
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-          if (k + u < k1) v[u] = *reinterpret_cast<const uint4*>(rows + static_cast<uint32_t>(list[k + u]) * kRowBytes);
+        for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+      int count = 0;
+      for (int c = 0; c < n_list; c += 32) {
+        const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
+        unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(sl));
+        count += __popc(mask);
+        while (mask) {
+          int tok[R];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (k + u < k1) {
-            float f[8];
-            Vec16<__nv_bfloat16>::unpack(v[u], f);
+          for (int r = 0; r < R; ++r) {
+            tok[r] = -1;
+            if (mask) {
+              const int l = __ffs(mask) - 1;
+              mask &= mask - 1;
+              tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
+            }
+          }
+          uint4 raw[R][VPL];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[e] += f[e];
+          for (int r = 0; r < R; ++r) {
+            const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+              const int v = v0 + lane + 32 * i;
+              if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
+            }
+          }
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            if (tok[r] < 0) continue;
+#pragma unroll
+            for (int i = 0; i < VPL; ++i) {
+              const int v = v0 + lane + 32 * i;
+              if (v < vecs) {
+                float f[E];
+                Vec16<__nv_bfloat16>::unpack(raw[r][i], f);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+              }
+            }
           }
         }
       }
-      const int count = k1 - k0;
       const float inv = 1.f / static_cast<float>(max(count, 1));
-      if (col < m.dim) {
-        float f[8];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) f[e] = acc[e] * inv;
-        st_16(static_cast<__nv_bfloat16*>(m.merged) + (static_cast<size_t>(b) * m.n_kept + sl) * m.dim + col,
-              Vec16<__nv_bfloat16>::pack(f));
+      for (int i = 0; i < VPL; ++i) {
+        const int v = v0 + lane + 32 * i;
+        if (v < vecs) {
+          float f[E];
+#pragma unroll
+          for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
+          st_16(reinterpret_cast<uint4*>(out) + v, Vec16<__nv_bfloat16>::pack(f));
+        }
       }
-      if (slice == 0 && piece == 0 && m.counts) m.counts[static_cast<size_t>(b) * m.n_kept + sl] = count;
+      if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
     }
-    __syncthreads();   // every thread has read the slice: the next one may overwrite it
   }
 }
 
-template <int kMinCtas>
-__global__ void __launch_bounds__(kThreads, kMinCtas)
-merge_interleaved_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                         const __grid_constant__ CUtensorMap map_x, Params p, Interleave il) {
-  extern __shared__ unsigned char smem_dyn[];
-  __shared__ Shared sh;
-  __shared__ MeanShared ms;
-  const int n_assign = p.m.instances * il.tiles, bid = blockIdx.x;
-  int mean_b, part;
-  if (bid < n_assign) {
-    const int b = bid / il.tiles;
-    part = bid - b * il.tiles;
-    assign_tile(&map_a, &map_b, p, sh, smem_dyn, b, part * kTileM, il.done + b);
-    mean_b = b - il.lag;
-    if (mean_b < 0) return;
-    __syncthreads();   // the tile's teardown is complete: shared memory changes hands
-  } else {
-    const int r = bid - n_assign;
-    mean_b = p.m.instances - il.lag + r / il.tiles;
-    part = r - (r / il.tiles) * il.tiles;
-    // A CTA of a kernel that uses tensor memory keeps the right to allocate it until it gives that right
-    // up, and the SM starts no further CTA of the kernel beside it meanwhile: take the smallest
-    // allocation and relinquish at once, as the assignment CTAs do.
-    if (threadIdx.x < 32) {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ms.tmem_base)), "r"(32) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    grid_dependency_launch();
-    grid_dependency_wait();   // the features may come from the kernel before this one
+// Packs the kept rows like pack_kept_kernel and, having read them anyway, writes 1 / max(|m_s|, eps) of every
+// kept token; the first CTA also zeroes the status word and the counters of the persistent kernel that
+// follows.  One warp per slot, the whole row in flight at once.
+__global__ void __launch_bounds__(256) pack_kept_norm_kernel(MergeParams m, int rows_packed) {
+  grid_dependency_launch();
+  if (blockIdx.x == 0 && blockIdx.y == 0) {
+    if (threadIdx.x == 0) *m.status = 0u;
+    for (int i = threadIdx.x; i <= m.instances; i += 256) m.counters[i] = 0;
   }
-  mean_share(&map_x, p.m, il, ms, smem_dyn, mean_b, part);
-  if (bid >= n_assign) {
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(ms.tmem_base), "r"(32) : "memory");
+  const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (s >= rows_packed) return;
+  uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.kept_packed) +
+                                        (static_cast<size_t>(b) * rows_packed + s) * m.metric_dim);
+  const int vecs = m.metric_dim / 8;
+  if (s >= m.n_kept) {
+    for (int v = lane; v < vecs; v += 32) st_16(dst + v, make_uint4(0u, 0u, 0u, 0u));
+    return;
+  }
+  grid_dependency_wait();   // the kept list comes from the kernel before this one
+  const int t = min(max(m.kept[static_cast<size_t>(b) * m.n_kept + s], 0), m.n_tokens - 1);
+  const uint4* src = reinterpret_cast<const uint4*>(
+      static_cast<const __nv_bfloat16*>(m.metric) + (static_cast<size_t>(b) * m.row_len + m.cls_offset + t) * m.metric_dim);
+  float ss = 0.f;
+  for (int v0 = 0; v0 < vecs; v0 += 128) {
+    uint4 r[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) { const int v = v0 + lane + 32 * u; if (v < vecs) r[u] = ld_nc_16(src + v); }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int v = v0 + lane + 32 * u;
+      if (v < vecs) {
+        st_16(dst + v, r[u]);
+        float f[8];
+        Vec16<__nv_bfloat16>::unpack(r[u], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) ss = fmaf(f[e], f[e], ss);
+      }
     }
+  }
+  ss = warp_sum(ss);
+  if (lane == 0) m.inv_norm[static_cast<size_t>(b) * m.n_kept + s] = 1.f / fmaxf(sqrtf(ss), 1e-12f);
+}
+
+// dynamic shared memory: alignment slack | stages x [A tile | B tile] | inv_norm[2][n_pad] | list and staged
+// assignments of the mean group (2 * n_tokens words)
+__global__ void __launch_bounds__(kPersistThreads, 1)
+merge_persistent_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p,
+                        Persist ps) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ PersistShared shp;
+  Shared& sh = shp.a;
+  unsigned char* tiles = smem_dyn + ((1024u - (smem_u32(smem_dyn) & 1023u)) & 1023u);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const MergeParams& m = p.m;
+  volatile int* abort_flag = &sh.abort_flag;
+  const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
+  float* inv_norm = reinterpret_cast<float*>(tiles + p.stages * stage_bytes);   // [accumulator][n_pad]
+  uint32_t* mean_list = reinterpret_cast<uint32_t*>(inv_norm + 2 * p.n_pad);
+
+  if (threadIdx.x == 0) {
+    // a stage is free again once the MMAs that read it have completed (the norms of the kept rows come
+    // from the packing kernel, so the read-back warps never touch the stages)
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 4); }
+    sh.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = sh.tmem_base;
+  grid_dependency_launch();
+  grid_dependency_wait();   // packed kept rows, norms and cleared counters come from the kernel before this one
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    const int groups = p.n_pad / 4;
+    int it = 0, cur_b = -1;
+    int rows[2][4];
+    bool ok = true;
+    for (int w = blockIdx.x; w < ps.total_tiles && ok; w += gridDim.x) {
+      const int b = w / ps.tiles, t0 = (w - b * ps.tiles) * kTileM;
+      if (b != cur_b) {   // row coordinates of the instance's kept tokens; padding repeats the first one
+        const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
+        const int row_base = b * m.row_len + m.cls_offset;
+        const int first = row_base + min(max(kept[0], 0), m.n_tokens - 1);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int g = lane + 32 * i;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int s_idx = g * 4 + j;
+            rows[i][j] = (g < groups && s_idx < m.n_kept) ? row_base + min(max(kept[s_idx], 0), m.n_tokens - 1) : first;
+          }
+        }
+        cur_b = b;
+      }
+      for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++it) {
+        const int s = it % p.stages, round = it / p.stages;
+        if (round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
+        if (!ok) break;
+        unsigned char* at = tiles + s * stage_bytes;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes + p.n_pad * 128);
+          tma_load_3d(at, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
+          if (p.b_packed) tma_load_3d(at + p.a_stage_bytes, &map_b, &sh.full[s], kc * kChunkK, 0, b);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const int g = lane + 32 * i;
+          if (g < groups && !p.b_packed)
+            tma_gather4(at + p.a_stage_bytes + g * 512, &map_b, &sh.full[s], kc * kChunkK, rows[i][0], rows[i][1],
+                        rows[i][2], rows[i][3]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = instr_desc_bf16(p.n_pad);
+      int it = 0, i = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < ps.total_tiles && ok && !*abort_flag; w += gridDim.x, ++i) {
+        const int acc = i & 1, use = i >> 1;
+        if (use > 0) {
+          if (!mbar_wait(&sh.tmem_empty[acc], (use - 1) & 1, abort_flag)) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        const uint32_t d_addr = tmem_acc + acc * p.n_pad;
+        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+          const int s = it % p.stages, round = it / p.stages;
+          if (!mbar_wait(&sh.full[s], round & 1, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = smem_u32(tiles + s * stage_bytes), b_addr = a_addr + p.a_stage_bytes;
+          const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
+#pragma unroll
+          for (int k = 0; k < kChunkK / 16; ++k) umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
+          umma_commit(&sh.empty[s]);
+        }
+        if (ok) umma_commit(&sh.tmem_full[acc]);
+      }
+    }
+    __syncwarp();
+  } else if (warp < kThreads / 32) {
+    // ------------------------------------------------------------ read-back: accumulator -> arg-max -> assignments
+    const int ptid = (warp - 2) * 32 + lane;  // 0..127
+    const int quarter = warp & 3;             // tensor-memory lanes this warp may read
+    const int row = quarter * 32 + lane;      // token row of this thread within the tile
+    int i = 0;
+    bool ok = true;
+    // Once `ok` drops the loops keep running with their work skipped, so that the four warps execute
+    // the same sequence of named barriers and warp-wide instructions whatever happens.
+    for (int w = blockIdx.x; w < ps.total_tiles; w += gridDim.x, ++i) {
+      const int b = w / ps.tiles, t0 = (w - b * ps.tiles) * kTileM;
+      const int acc = i & 1, use = i >> 1;
+      const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
+      // 1 / |m_s| of the instance's kept tokens -> shared memory; this buffer was last read two tiles ago,
+      // before that tile's arrive on tmem_empty
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int r = ptid + 128 * u;
+        if (r < p.n_pad) inv_norm[acc * p.n_pad + r] = (r < m.n_kept) ? __ldcg(m.inv_norm + static_cast<size_t>(b) * m.n_kept + r) : 0.f;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
+      float best_val = -INFINITY;
+      int best_idx = 0;
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.n_pad;
+        for (int c0 = 0; c0 < p.n_pad; c0 += 32) {
+          uint32_t v[32];
+          if (p.n_pad - c0 >= 32) tmem_ld32(taddr + c0, v);
+          else {
+            tmem_ld16(taddr + c0, v);
+#pragma unroll
+            for (int j = 16; j < 32; ++j) v[j] = 0u;
+          }
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (c0 + j < p.n_pad && c0 + j < m.n_kept) {
+              const float val = __uint_as_float(v[j]) * inv_norm[acc * p.n_pad + c0 + j];
+              if (val > best_val) { best_val = val; best_idx = c0 + j; }
+            }
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.tmem_empty[acc]);
+      }
+      sh.best_slot[row] = best_idx;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      // a kept token belongs to its own slot
+      for (int s_idx = ptid; s_idx < m.n_kept; s_idx += 128) {
+        const int t = min(max(kept[s_idx], 0), m.n_tokens - 1);
+        if (t >= t0 && t < t0 + kTileM) sh.best_slot[t - t0] = s_idx;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok && t0 + ptid < m.n_tokens) m.assign[static_cast<size_t>(b) * m.n_tokens + t0 + ptid] = sh.best_slot[ptid];
+      // publish: the stores above first, then one increment of the instance's counter
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ptid == 0 && ok && !*abort_flag) atomicAdd(ps.done + b, 1);
+    }
+  } else {
+    // ------------------------------------------------------------ mean group
+    const int gtid = threadIdx.x - kThreads;
+    while (true) {
+      if (gtid == 0) {
+        const int q = atomicAdd(ps.job_head, 1);
+        int ready = 1;
+        if (q < ps.total_jobs) {
+          const volatile int* flag = ps.done + q / ps.jobs_per_instance;
+          uint32_t spins = 0;
+          while (*flag < ps.tiles && spins < kDoneSpinLimit && !*abort_flag) { __nanosleep(100); ++spins; }
+          ready = *flag >= ps.tiles;
+          if (!ready) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+          __threadfence();
+        }
+        shp.job = q;
+        shp.ready = ready;
+      }
+      mean_group_sync();
+      const int q = shp.job, ready = shp.ready;
+      mean_group_sync();   // everyone has the job before thread 0 takes the next one
+      if (q >= ps.total_jobs || !ready) break;
+      mean_job<4, 4>(m, q / ps.jobs_per_instance, (q % ps.jobs_per_instance) * kJobSlots, mean_list, shp.warp_sums, gtid);
+    }
+  }
+
+  // ------------------------------------------------------------ teardown
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (sh.abort_flag) {
+    if (threadIdx.x == 0) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);   // copies still in flight land before the memory is released
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(p.tmem_cols) : "memory");
   }
 }
 
@@ -563,7 +782,7 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   return VSCAN_OK;
 }
 
-// ---- assignment + group means in one launch
+// ---- assignment + group means in one persistent launch
 static int sm_count() {
   static int n = 0;
   if (n == 0) {
@@ -574,71 +793,57 @@ static int sm_count() {
   return n;
 }
 
-static bool plan_interleaved(const MergeParams& m, tc::Params& p, tc::Interleave& il, int& ctas_per_sm, size_t& smem) {
-  if (!tc::plan(m, p) || p.n_chunks != 1 || p.b_packed) return false;
-  const int stage = p.a_stage_bytes + p.b_stage_bytes;
-  ctas_per_sm = (73 * 1024) / stage >= 3 ? 3 : ((110 * 1024) / stage >= 3 ? 2 : 1);
-  smem = tc::smem_bytes(p);
-  // the sums: the column slice of every token (whole tile loads) + the member list
-  il.x_boxes = (m.n_tokens + tc::kBoxRows - 1) / tc::kBoxRows;
-  if (il.x_boxes > tc::kMaxBoxes || m.n_kept > tc::kMaxMeanKept) return false;
-  const size_t slice_bytes = static_cast<size_t>(il.x_boxes) * tc::kBoxRows * tc::kSliceCols * 2;
-  if (128 + slice_bytes + static_cast<size_t>(m.n_tokens) * 2 > smem) return false;
-  if (static_cast<size_t>(m.n_kept) * ((m.n_tokens + 31) / 32) * 6 > slice_bytes) return false;   // the sort's scratch
-  if ((reinterpret_cast<uintptr_t>(m.x) & 15u) != 0 || m.dim % 8 != 0) return false;
-  il.done = reinterpret_cast<int*>(m.inv_norm);   // the tensor path takes the norms itself: the region is free
-  il.tiles = (m.n_tokens + tc::kTileM - 1) / tc::kTileM;
-  il.slices = (m.dim + tc::kSliceCols - 1) / tc::kSliceCols;
-  // far enough back that the instance's tiles have finished, near enough that its features are still in L2
-  int lag = 16;
-  if (const char* e = getenv("VSCAN_MERGE_LAG")) lag = atoi(e) > 0 ? atoi(e) : lag;
-  il.lag = lag < m.instances ? lag : m.instances;
-  if ((static_cast<long long>(m.instances) + il.lag) * il.tiles > 0x7fffffffLL) return false;
+static bool plan_persistent(const MergeParams& m, tc::Params& p, tc::Persist& ps, size_t& smem) {
+  if (!tc::plan(m, p) || p.n_chunks != 1 || p.b_packed || m.kept_packed == nullptr) return false;
+  p.b_packed = 1;   // one producer warp per SM: a tile load of the packed kept rows per stage instead of n_pad / 4 row gathers
+  if (m.counters == nullptr || m.inv_norm == nullptr) return false;
+  if ((reinterpret_cast<uintptr_t>(m.x) & 15u) != 0 || m.dim % 8 != 0 || m.n_tokens >= (1 << 24)) return false;
+  // one CTA per SM: as many stages as fit beside the inverse norms (two accumulators) and the mean group's lists
+  const size_t stage = static_cast<size_t>(p.a_stage_bytes + p.b_stage_bytes);
+  const size_t fixed = 1024 + 2 * static_cast<size_t>(p.n_pad) * sizeof(float) + static_cast<size_t>(m.n_tokens) * 8 + 16;
+  if (fixed + 3 * stage > 224 * 1024) return false;
+  size_t stages = (224 * 1024 - fixed) / stage;
+  if (stages > tc::kMaxStages) stages = tc::kMaxStages;
+  p.stages = static_cast<int>(stages);
+  p.tmem_cols = 32;
+  while (p.tmem_cols < 2 * p.n_pad) p.tmem_cols *= 2;
+  smem = fixed + stages * stage;
+  ps.done = m.counters;
+  ps.job_head = ps.done + m.instances;
+  ps.tiles = (m.n_tokens + tc::kTileM - 1) / tc::kTileM;
+  const long long total_tiles = static_cast<long long>(m.instances) * ps.tiles;
+  ps.jobs_per_instance = (m.n_kept + tc::kJobSlots - 1) / tc::kJobSlots;
+  const long long total_jobs = static_cast<long long>(m.instances) * ps.jobs_per_instance;
+  if (total_tiles > 0x3fffffffLL || total_jobs > 0x3fffffffLL) return false;
+  ps.total_tiles = static_cast<int>(total_tiles);
+  ps.total_jobs = static_cast<int>(total_jobs);
   return true;
 }
 
 bool merge_interleaved_supported(int dtype, const MergeParams& m) {
   if (!assign_tensor_supported(dtype, m)) return false;
-  tc::Params p; tc::Interleave il; int c; size_t smem;
-  return plan_interleaved(m, p, il, c, smem);
+  tc::Params p; tc::Persist ps; size_t smem;
+  return plan_persistent(m, p, ps, smem);
 }
 
 vscan_status launch_merge_interleaved(const MergeParams& m_in, cudaStream_t stream) {
   MergeParams m = m_in;
-  m.clear_status = 0;   // the memset below clears the status word together with the counters
-  tc::Params p; tc::Interleave il; int ctas_per_sm; size_t smem;
-  if (!plan_interleaved(m, p, il, ctas_per_sm, smem)) return VSCAN_ERR_UNSUPPORTED;
-  CUtensorMap map, map_b, map_x;
+  m.clear_status = 0;   // the packing kernel clears the status word together with the counters
+  tc::Params p; tc::Persist ps; size_t smem;
+  if (!plan_persistent(m, p, ps, smem)) return VSCAN_ERR_UNSUPPORTED;
+  CUtensorMap map, map_b;
   vscan_status st = encode_maps(m, p, map, map_b);
   if (st != VSCAN_OK) return st;
-  {   // column slices of the features for the sums: [instance][row][dim], box = kSliceCols columns x kBoxRows rows
-    const cuuint64_t dims[3] = {static_cast<cuuint64_t>(m.dim), static_cast<cuuint64_t>(m.row_len),
-                                static_cast<cuuint64_t>(m.instances)};
-    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(m.dim) * 2, static_cast<cuuint64_t>(m.row_len) * m.dim * 2};
-    const cuuint32_t box[3] = {tc::kSliceCols, tc::kBoxRows, 1};
-    const cuuint32_t elem[3] = {1, 1, 1};
-    if (tc::encode_fn()(&map_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(m.x), dims, strides, box, elem,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return VSCAN_ERR_UNSUPPORTED;
+  {   // packed kept rows + their inverse norms; also clears the status word and the counters
+    dim3 pgrid((static_cast<unsigned>(p.n_pad) + 7) / 8, m.instances);
+    VSCAN_LAUNCH("pack_kept", stream,
+                 (void)launch_dependent(tc::pack_kept_norm_kernel, pgrid, dim3(256), 0, stream, m, p.n_pad));
   }
-  // status word (first 256 bytes of the workspace) and the counters right behind it
-  if (reinterpret_cast<char*>(il.done) != reinterpret_cast<char*>(m.status) + kStatusBytes) return VSCAN_ERR_WORKSPACE;
-  VSCAN_CUDA_TRY(cudaMemsetAsync(m.status, 0, kStatusBytes + static_cast<size_t>(m.instances) * sizeof(int), stream));
-  const unsigned blocks = static_cast<unsigned>(m.instances + il.lag) * il.tiles;
-  if (ctas_per_sm == 3) {
-    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<3>, smem));
-    VSCAN_LAUNCH("merge_interleaved", stream,
-                 (void)launch_dependent(tc::merge_interleaved_kernel<3>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
-  } else if (ctas_per_sm == 2) {
-    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<2>, smem));
-    VSCAN_LAUNCH("merge_interleaved", stream,
-                 (void)launch_dependent(tc::merge_interleaved_kernel<2>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
-  } else {
-    VSCAN_CUDA_TRY(allow_smem(tc::merge_interleaved_kernel<1>, smem));
-    VSCAN_LAUNCH("merge_interleaved", stream,
-                 (void)launch_dependent(tc::merge_interleaved_kernel<1>, dim3(blocks), dim3(tc::kThreads), smem, stream, map, map_b, map_x, p, il));
-  }
+  const int sms = sm_count();
+  const unsigned blocks = static_cast<unsigned>(ps.total_tiles < sms ? ps.total_tiles : sms);
+  VSCAN_CUDA_TRY(allow_smem(tc::merge_persistent_kernel, smem));
+  VSCAN_LAUNCH("merge_persistent", stream,
+               (void)launch_dependent(tc::merge_persistent_kernel, dim3(blocks), dim3(tc::kPersistThreads), smem, stream, map, map_b, p, ps));
   return VSCAN_OK;
 }
 
