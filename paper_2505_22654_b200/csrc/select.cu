@@ -180,7 +180,12 @@ static void fill_params(SelectParams& p, const vscan_select_desc* d, long long n
 }
 
 // One warp per window while there are enough windows to fill the block.
-static int select_threads(long long n, int windows) { return n > 2048 ? 1024 : (windows > 8 || n > 256 ? 512 : 256); }
+static int select_threads(long long n, int windows) {
+  if (n > 2048) return 1024;
+  // a thread per token where that is possible, so that the scores of an instance are read in one round of loads
+  if (n > 512 && n <= 1024) return static_cast<int>((n + 31) / 32 * 32);
+  return windows > 8 || n > 256 ? 512 : 256;
+}
 
 extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
                                                   size_t /*workspace_bytes*/, void* stream) {
