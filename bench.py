@@ -31,7 +31,7 @@ from synth import CONFIGS, stage1_inputs, stage2_inputs, sweep_config  # noqa: E
 METRIC = "VScan reduction images/s (Stage1+Stage2) at 2880 visual tokens"
 UNIT = "images/s"
 FALLBACK_HBM_GBS = 6650.0
-MERGE_KERNELS = ("kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", "merge_fused", "merge_persistent")
+MERGE_KERNELS = ("kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", "merge_fused", "merge_persistent", "pack_kept")
 
 
 # ------------------------------------------------------------------ algorithmic work per step
