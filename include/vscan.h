@@ -277,6 +277,17 @@ vscan_status vscan_check(const void* workspace, void* stream);
 int32_t vscan_last_cuda_error(void);
 uint64_t vscan_kernel_launches(void);
 
+/* ---------------------------------------------------------------------------------------------
+ * vscan_selftest_bounded_wait: exercises the failure path of the device-side waits without touching any
+ * data.  Visual rows of the Stage-2 compaction wait for their sequence's survivor list (Sec. 4.2, the
+ * KV-cache remark: only survivors are moved) with a bound on the number of polls; when the bound runs out
+ * the CTA records VSCAN_ERR_TIMEOUT in the status word and returns, and the context stays usable.  This call
+ * launches one CTA that waits in the same way, `polls` polls of about 100 ns (1 .. 2^24), on a flag that
+ * nothing sets; vscan_check(workspace, stream) must then return VSCAN_ERR_TIMEOUT.
+ *   workspace  device memory, 256-byte aligned, at least 512 bytes; its first 512 bytes are overwritten.
+ * ------------------------------------------------------------------------------------------- */
+vscan_status vscan_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t polls, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

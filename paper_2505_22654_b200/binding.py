@@ -92,6 +92,8 @@ def lib() -> C.CDLL:
         L.vscan_profile_begin.restype, L.vscan_profile_begin.argtypes = _i32, [_i32]
         L.vscan_profile_end.restype = _i32
         L.vscan_profile_end.argtypes = [C.c_char_p, C.POINTER(C.c_float), _i32]
+        L.vscan_selftest_bounded_wait.restype = _i32
+        L.vscan_selftest_bounded_wait.argtypes = [_vp, C.c_size_t, C.c_uint32, _vp]
         L.vscan_score_qk_static_capacity.restype = C.c_size_t
         L.vscan_score_qk_static.restype = _i32
         L.vscan_score_qk_static.argtypes = [C.POINTER(ScoreDesc), _vp]
@@ -322,3 +324,11 @@ def profile_end(capacity: int = 4096):
 
 def vscan_check(workspace: Workspace) -> int:
     return int(lib().vscan_check(workspace.ptr, _stream()))
+
+
+def vscan_selftest_bounded_wait(workspace: Workspace, polls: int = 2000) -> None:
+    """One CTA waits `polls` polls on a flag nothing sets; vscan_check(workspace) then reports the timeout."""
+    workspace.reserve(512)
+    st = lib().vscan_selftest_bounded_wait(workspace.ptr, C.c_size_t(workspace.buf.numel()), C.c_uint32(polls), _stream())
+    if st != 0:
+        raise VScanError(st, "vscan_selftest_bounded_wait")

@@ -161,6 +161,14 @@ __device__ __forceinline__ void st_16(void* p, const uint4& r) {
                : "memory");
 }
 
+// Bounded spin on a flag that another CTA sets (polls about 100 ns apart).  Returns true once *flag >= target,
+// false when `limit` polls have gone by; the caller then records VSCAN_ERR_TIMEOUT and leaves.
+__device__ __forceinline__ bool wait_flag_bounded(const volatile int* flag, int target, unsigned limit) {
+  unsigned spins = 0;
+  while (*flag < target && spins < limit) { __nanosleep(100); ++spins; }
+  return *flag >= target;
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

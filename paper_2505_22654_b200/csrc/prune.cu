@@ -130,10 +130,7 @@ __global__ void __launch_bounds__(kPruneThreads) prune_fused_kernel(QkParams q, 
   if (dependent) {
     __shared__ int ok;
     if (threadIdx.x == 0) {
-      unsigned spins = 0;
-      const volatile int* flag = q.ready + b;
-      while (*flag == 0 && spins < kReadySpinLimit) { __nanosleep(100); ++spins; }
-      ok = *flag != 0;
+      ok = wait_flag_bounded(q.ready + b, 1, kReadySpinLimit);
       if (!ok && q.status) atomicExch(q.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
       __threadfence();
     }
@@ -163,9 +160,25 @@ static vscan_status launch_prune_fused(const QkParams& q, const CompactParams& c
 #undef VSCAN_PRUNE_CASE
 }
 
+// One CTA that waits, the way a row-copy CTA waits for its sequence's survivor list, on a flag nobody sets.
+__global__ void __launch_bounds__(32) selftest_wait_kernel(uint32_t* status, int* flag, unsigned limit) {
+  if (threadIdx.x == 0 && !wait_flag_bounded(flag, 1, limit)) atomicExch(status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+}
+
 }  // namespace vscan
 
 using namespace vscan;
+
+extern "C" vscan_status vscan_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t polls, void* stream_) {
+  if (!workspace || !aligned256(workspace) || workspace_bytes < 2 * kStatusBytes) return VSCAN_ERR_WORKSPACE;
+  if (polls == 0 || polls > (1u << 24)) return VSCAN_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  VSCAN_CUDA_TRY(cudaMemsetAsync(workspace, 0, 2 * kStatusBytes, stream));   // status word and the flag
+  int* flag = reinterpret_cast<int*>(static_cast<char*>(workspace) + kStatusBytes);
+  VSCAN_LAUNCH("selftest_wait", stream,
+               (selftest_wait_kernel<<<1, 32, 0, stream>>>(static_cast<uint32_t*>(workspace), flag, polls)));
+  return VSCAN_OK;
+}
 
 static vscan_status validate_prune(const vscan_prune_desc* d) {
   if (!d || !d->q_last || !d->k || !d->k_out) return VSCAN_ERR_INVALID_ARG;

@@ -361,3 +361,20 @@ def test_workspace_too_small_and_status_word():
     vs.vscan_llm_prune(*args, workspace=ws)
     assert vs.vscan_check(ws) == 0
     assert vs.kernel_launches() > 0
+
+
+# ------------------------------------------------------------------ failure path of the device-side waits
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """A wait on a flag that nothing sets gives up after its bound, the status word says so, and the
+    context is still usable: the next call on the same workspace succeeds and clears the status."""
+    ws = vs.Workspace(8 << 20)
+    vs.vscan_selftest_bounded_wait(ws, polls=2000)          # about 0.2 ms
+    assert vs.vscan_check(ws) == 5                          # VSCAN_ERR_TIMEOUT
+    assert vs.status_string(5)
+    x = torch.randn((1, 40, 16), device="cuda")
+    kept = torch.tensor([[1, 5]], dtype=torch.int32, device="cuda")
+    merged = vs.vscan_merge(x, 0, kept, workspace=ws)
+    assert vs.vscan_check(ws) == 0
+    assert torch.isfinite(merged).all()
+    with pytest.raises(vs.VScanError):
+        vs.vscan_selftest_bounded_wait(ws, polls=0)
