@@ -158,6 +158,24 @@ __global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergePara
   group_mean_body<T, VPL, R, kSlotsPerCta>(p, blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums);
 }
 
+template <typename T, int VPL, int R>
+__global__ void __launch_bounds__(128) group_mean_bits_kernel(MergeParams p) {
+  extern __shared__ __align__(16) unsigned char smem_bits[];
+  grid_dependency_wait();   // the assignments come from the kernel before this one
+  group_mean_bits_body<T, VPL, R>(p, blockIdx.y, blockIdx.x * 4, smem_bits);
+}
+
+template <typename T, int VPL, int R>
+static vscan_status launch_group_mean_bits(const MergeParams& p, cudaStream_t stream) {
+  const size_t chunks = (static_cast<size_t>(p.n_tokens) + 31) / 32;
+  const size_t smem = 4 * chunks * 4 + 4 * static_cast<size_t>(p.n_tokens) * 2 + 16;
+  dim3 grid((p.n_kept + 3) / 4, p.instances);
+  VSCAN_CUDA_TRY(allow_smem(group_mean_bits_kernel<T, VPL, R>, smem));
+  VSCAN_LAUNCH("group_mean", stream,
+               (void)launch_dependent(group_mean_bits_kernel<T, VPL, R>, grid, dim3(128), smem, stream, p));
+  return VSCAN_OK;
+}
+
 template <typename T, int VPL, int R, int SLOTS>
 static vscan_status launch_group_mean_as(const MergeParams& p, size_t smem, cudaStream_t stream) {
   dim3 grid((p.n_kept + SLOTS - 1) / SLOTS, p.instances);
@@ -176,7 +194,7 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   // 512-thread CTAs have 128 registers per thread: wide rows are then summed in two column passes
   // (4 pieces per lane each) rather than with 8 pieces per lane, which would spill
   if (long_instance) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
-  if (!wide) return launch_group_mean_as<T, 2, 4, 4>(p, smem, stream);   // two column passes, 56 registers: more CTAs per SM
+  if (!wide) return launch_group_mean_bits<T, 2, 4>(p, stream);   // two column passes, few registers: more CTAs per SM
   return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
 }
 

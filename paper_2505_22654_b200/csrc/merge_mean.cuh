@@ -120,3 +120,116 @@ __device__ __forceinline__ void group_mean_body(const MergeParams& p, int b, int
 
 
 }  // namespace vscan
+
+namespace vscan {
+
+// Short instances: the same sums with a cheaper prologue.  Four slots per CTA, warp w owns slot s0 + w.
+// Every thread marks its tokens in a bit mask per (slot, 32-token chunk) with shared-memory atomics (two
+// block barriers in all, no scan); warp w then turns the masks of its slot into its own list of members
+// (ascending token order: chunk by chunk, bit by bit) with one warp-wide prefix sum, and walks it with R
+// rows in flight.  Same order of additions as group_mean_body, hence the same bits.
+// dynamic shared memory: bits[4][chunks] words | lists[4][n_tokens] halfwords.  n_tokens < 65536.
+template <typename T, int VPL, int R>
+__device__ __forceinline__ void group_mean_bits_body(const MergeParams& p, int b, int s0, unsigned char* smem) {
+  constexpr int E = Vec16<T>::kElems;
+  constexpr int kSlots = 4, kThreadsCta = kSlots * 32;
+  const int chunks = (p.n_tokens + 31) / 32;
+  uint32_t* bits = reinterpret_cast<uint32_t*>(smem);
+  uint16_t* lists = reinterpret_cast<uint16_t*>(bits + kSlots * chunks);
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int i = threadIdx.x; i < kSlots * chunks; i += kThreadsCta) bits[i] = 0u;
+  __syncthreads();
+  {
+    const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
+    for (int i0 = threadIdx.x; i0 < p.n_tokens; i0 += kThreadsCta * 8) {
+      int32_t v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kThreadsCta; v[u] = i < p.n_tokens ? __ldcg(ag + i) : -1; }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * kThreadsCta;
+        const unsigned rel = static_cast<unsigned>(v[u] - s0);
+        if (i < p.n_tokens && rel < static_cast<unsigned>(kSlots)) atomicOr(&bits[rel * chunks + (i >> 5)], 1u << (i & 31));
+      }
+    }
+  }
+  __syncthreads();
+  const int s = s0 + w;
+  if (s >= p.n_kept) return;
+  // the members of slot s: lane l expands the mask words l, l + 32, ... in order
+  uint16_t* list = lists + static_cast<size_t>(w) * p.n_tokens;
+  int count = 0;
+  for (int c0 = 0; c0 < chunks; c0 += 32) {
+    const int c = c0 + lane;
+    uint32_t word = c < chunks ? bits[w * chunks + c] : 0u;
+    const int mine = __popc(word);
+    int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    int pos = count + incl - mine;
+    while (word) {
+      const int bit = __ffs(word) - 1;
+      word &= word - 1;
+      list[pos++] = static_cast<uint16_t>(c * 32 + bit);
+    }
+    count += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  __syncwarp();
+
+  const int vecs = p.dim / E;
+  const T* xb = static_cast<const T*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
+  T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
+  for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
+    float acc[VPL][E];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+    for (int k = 0; k < count; k += R) {
+      uint4 raw[R][VPL];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (k + r < count) {
+          const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(list[k + r]) * p.dim);
+#pragma unroll
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs) raw[r][i] = ld_nc_16(row + v);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (k + r < count) {
+#pragma unroll
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs) {
+              float f[E];
+              Vec16<T>::unpack(raw[r][i], f);
+#pragma unroll
+              for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+            }
+          }
+        }
+      }
+    }
+    const float inv = 1.f / static_cast<float>(max(count, 1));
+#pragma unroll
+    for (int i = 0; i < VPL; ++i) {
+      const int v = v0 + lane + 32 * i;
+      if (v < vecs) {
+        float f[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
+        st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
+      }
+    }
+    if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
+  }
+}
+
+}  // namespace vscan
