@@ -36,9 +36,17 @@ __device__ __forceinline__ void block_radix_select(const uint32_t* keys, const u
         const int i = base + threadIdx.x;
         const bool valid = i < n && !(excluded && excluded[i]);
         const uint32_t digit = valid ? (keys[i] >> 24) : 0u;
+        // the lanes that share the digit of the warp's first candidate are counted with one atomic, the
+        // others (few) add one by one
         const unsigned lane = threadIdx.x & 31;
-        const unsigned peers = __match_any_sync(0xffffffffu, valid ? digit : (256u + lane));
-        if (valid && lane == static_cast<unsigned>(__ffs(peers) - 1)) atomicAdd(&sc.hist[digit], __popc(peers));
+        const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+        if (vmask) {
+          const int lead = __ffs(vmask) - 1;
+          const uint32_t d0 = __shfl_sync(0xffffffffu, digit, lead);
+          const unsigned same = __ballot_sync(0xffffffffu, valid && digit == d0);
+          if (lane == static_cast<unsigned>(lead)) atomicAdd(&sc.hist[d0], __popc(same));
+          if (valid && digit != d0) atomicAdd(&sc.hist[digit], 1);
+        }
       }
     } else {
       for (int i = threadIdx.x; i < n; i += blockDim.x) {
