@@ -253,7 +253,8 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
     n_sets = args.sets
     warmup = max(args.warmup, 3)
     sets = build_sets(cfg, n_sets, device)
-    reducers = [vs.VScanReducer.from_config(cfg, device=device, merge_path=args.merge_path) for _ in range(n_sets)]
+    reducers = [vs.VScanReducer.from_config(cfg, device=device, merge_path=args.merge_path,
+                                            overlap_stages=args.overlap_stages) for _ in range(n_sets)]
     stream = torch.cuda.Stream(device)
     launches_per_step = 0
     with torch.cuda.stream(stream):
@@ -451,6 +452,7 @@ def main():
     ap.add_argument("--sets", type=int, default=3, help="rotating buffer sets")
     ap.add_argument("--merge-path", type=int, default=0, help="0 auto, 1 CUDA cores, 2 tensor cores")
     ap.add_argument("--no-graph", action="store_true")
+    ap.add_argument("--overlap-stages", action="store_true", help="Stage 1 and Stage 2 as two parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="all named workloads and the batch x retention sweep")
     args = ap.parse_args()

@@ -86,6 +86,8 @@ typedef enum {
  *   scores    [batch][span_len] float32 (output).  head_dim must be a multiple of 8, at most 256;
  *             q_heads a multiple of kv_heads.
  * Fields of the mode not in use are ignored.  Workspace: QK mode only.
+ * Limits of this build (VSCAN_ERR_UNSUPPORTED, nothing enqueued): instances, batch <= 65535; QK mode:
+ * (head_dim + keys under the softmax) * 4 bytes must fit 227 KB of shared memory (about 58 000 keys).
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
   int32_t mode;  /* vscan_score_mode */
@@ -195,6 +197,8 @@ vscan_status vscan_score_select(const vscan_score_select_desc* desc, void* strea
  *             to its own slot).  When NULL it lives in the workspace.
  *   counts    optional [instances][n_kept] int32 output: group size including the kept token.
  * dim and metric_dim must be multiples of 8; 1 <= n_kept <= n_tokens.
+ * Limits of this build: n_tokens <= 29054 (one instance's member list is staged in shared memory),
+ * instances <= 65535; beyond them VSCAN_ERR_UNSUPPORTED, nothing enqueued.
  * `path` picks the unit for the similarity contraction (vscan_merge_path).
  * ------------------------------------------------------------------------------------------- */
 typedef struct {

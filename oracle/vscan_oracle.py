@@ -79,8 +79,8 @@ def received_attention(probs: np.ndarray) -> np.ndarray:
 
 # --------------------------------------------------------------------------- exact top-k
 def topk_lowest_index(scores: np.ndarray, k: int, candidates: np.ndarray | None = None) -> np.ndarray:
-    """The k candidates with the largest score; equal scores go to the lower index (Eq. 2: the
-    threshold tau "set to retain a target number of tokens").  Returns ascending indices.
+    """The k candidates with the largest score; equal scores go to the lower index (Sec. 4.1, text
+    after Eq. 2: the threshold tau is whatever value leaves the wanted count).  Returns ascending indices.
 
     A stable sort on descending score keeps equal scores in index order, so the first k entries
     are exactly the set {i : #{j : s_j > s_i or (s_j == s_i and j < i)} < k}.
@@ -162,13 +162,26 @@ def merge(x: np.ndarray, cls_offset: int, kept_idx: np.ndarray, metric: np.ndarr
     if unsel.size:
         cos = cosine_matrix(m[cls_offset + unsel], m[cls_offset + kept])
         assign[unsel] = np.argmax(cos, axis=1)       # first maximum: lowest slot on ties
+    merged, counts = mean_merge(x, cls_offset, kept, assign)
+    return merged, assign, counts
+
+
+def mean_merge(x: np.ndarray, cls_offset: int, kept_idx: np.ndarray, assign: np.ndarray):
+    """Eq. 4 alone, for groups that are already decided: assign[u] is the kept slot of token u (a kept
+    token holds its own slot).  merged[s] = (x_s + sum_{u in U^s} x_u) / (|U^s| + 1).
+    Returns merged [K1, D] float64 (unrounded) and counts [K1] (|U^s| + 1)."""
+    x = np.asarray(x, dtype=np.float64)
+    kept = np.asarray(kept_idx, dtype=np.int64)
+    N, K1 = x.shape[0] - cls_offset, kept.shape[0]
+    is_kept = np.zeros(N, dtype=bool)
+    is_kept[kept] = True
     merged = x[cls_offset + kept].copy()
     counts = np.ones(K1, dtype=np.int64)
-    for u in unsel:                                   # Eq. 4: sum over U^s, then divide
+    for u in np.nonzero(~is_kept)[0]:                 # sum over U^s in token order, then divide
         merged[assign[u]] += x[cls_offset + u]
         counts[assign[u]] += 1
     merged /= counts[:, None]
-    return merged, assign, counts
+    return merged, counts
 
 
 # --------------------------------------------------------------------------- Stage 2
@@ -227,19 +240,3 @@ def topk_boundary_gap(scores: np.ndarray, k: int, candidates: np.ndarray | None 
         return float("inf")
     v = np.sort(s[cand])[::-1]
     return float(v[k - 1] - v[k])
-
-
-def round_bf16(a: np.ndarray) -> np.ndarray:
-    """Round float64 values to the nearest bf16 (ties to even); returned as float64."""
-    f = np.asarray(a, dtype=np.float64).astype(np.float32)
-    # The two bf16 neighbours of the value (towards zero / away from zero) are compared in
-    # float64, so the intermediate float32 cast cannot cause a double rounding.
-    bits = f.view(np.uint32)
-    lo = (bits & np.uint32(0xFFFF0000)).view(np.float32).astype(np.float64)
-    hi_bits = ((bits & np.uint32(0xFFFF0000)) + np.uint32(0x00010000))
-    hi = hi_bits.view(np.float32).astype(np.float64)
-    a64 = np.asarray(a, dtype=np.float64)
-    dlo, dhi = np.abs(a64 - lo), np.abs(a64 - hi)
-    lo_even = ((bits >> np.uint32(16)) & np.uint32(1)) == 0
-    pick_lo = (dlo < dhi) | ((dlo == dhi) & lo_even)
-    return np.where(pick_lo, lo, hi)

@@ -2,6 +2,7 @@
 library is a plain shared object loaded with ctypes."""
 from __future__ import annotations
 
+import hashlib
 import os
 import shutil
 import subprocess
@@ -12,21 +13,41 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB_PATH = os.path.join(HERE, "libvscan.so")
 
+STAMP_PATH = LIB_PATH + ".digest"
+
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "--use_fast_math=false", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=default",
-              "-cudart", "static"]
+              "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=default", "-cudart", "static"]
 
 
 def sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
+def _deps():
+    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + [os.path.join(INCLUDE, "vscan.h")]
+
+
+def source_digest() -> str:
+    """Digest of everything the library is built from (file names and contents, build flags)."""
+    h = hashlib.sha256(" ".join(NVCC_FLAGS).encode())
+    for path in _deps():
+        h.update(os.path.basename(path).encode())
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
 def _stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+    """True when libvscan.so is missing or was built from other sources than the ones on disk.  The
+    digest recorded next to the library decides, not file times (a copied tree has arbitrary ones)."""
+    if not os.path.exists(LIB_PATH) or not os.path.exists(STAMP_PATH):
         return True
-    t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "vscan.h")]
-    return any(os.path.getmtime(d) > t for d in deps)
+    with open(STAMP_PATH) as f:
+        return f.read().strip() != source_digest()
+
+
+def have_nvcc() -> bool:
+    return os.path.exists(shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc")
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -36,14 +57,16 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = shutil.which("nvcc") or "/usr/local/cuda/bin/nvcc"
     if not os.path.exists(nvcc):
         raise RuntimeError("nvcc not found: libvscan.so cannot be built")
-    flags = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
-    cmd = [nvcc, "-shared", "-o", LIB_PATH, "-I", INCLUDE, "-I", CSRC] + flags
+    digest = source_digest()
+    cmd = [nvcc, "-shared", "-o", LIB_PATH, "-I", INCLUDE, "-I", CSRC] + NVCC_FLAGS
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources()
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    with open(STAMP_PATH, "w") as f:
+        f.write(digest + "\n")
     if verbose:
         sys.stderr.write(res.stderr)
     return LIB_PATH

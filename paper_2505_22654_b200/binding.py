@@ -67,12 +67,18 @@ _LIB = None
 
 
 def lib() -> C.CDLL:
-    """Load libvscan.so (building it first if the sources are newer).  Raises if unavailable."""
+    """Load libvscan.so, building it first when it is missing or was built from other sources than the
+    ones on disk.  Raises if it is unavailable, or stale with no compiler to rebuild it: a library that
+    does not match its sources is never loaded silently."""
     global _LIB
     if _LIB is None:
         path = _build.LIB_PATH
-        if not os.path.exists(path) or os.environ.get("VSCAN_REBUILD") == "1":
-            path = _build.build()
+        force = os.environ.get("VSCAN_REBUILD") == "1"
+        if force or _build._stale():
+            if not _build.have_nvcc():
+                raise RuntimeError(f"{path} is missing or does not match the sources under csrc/, and nvcc is "
+                                   "not available to rebuild it")
+            path = _build.build(force=force)
         L = C.CDLL(path)
         for name, desc in (("score", ScoreDesc), ("select", SelectDesc), ("merge", MergeDesc),
                            ("llm_prune", PruneDesc)):

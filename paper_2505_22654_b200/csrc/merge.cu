@@ -212,7 +212,8 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
       d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
     return VSCAN_ERR_INVALID_ARG;
   if (d->metric && (d->metric_dim <= 0 || d->metric_dim % 8)) return VSCAN_ERR_INVALID_ARG;
-  if (d->n_tokens >= (1 << 24)) return VSCAN_ERR_UNSUPPORTED;
+  // the group-mean kernels stage one instance's member list and assignments in shared memory
+  if (static_cast<size_t>(d->n_tokens) * 8 + 16 > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
   if (d->instances > 65535) return VSCAN_ERR_UNSUPPORTED;
   const void* ptrs[] = {d->x, d->metric, d->kept_idx, d->merged, d->assign, d->counts};
   for (const void* ptr : ptrs)

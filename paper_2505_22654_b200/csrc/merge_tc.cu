@@ -91,13 +91,15 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  if (m.clear_status && b == 0 && t0 == 0 && threadIdx.x == 0) *m.status = 0u;   // long before any wait can expire
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = sh.tmem_base;
   grid_dependency_launch();
   grid_dependency_wait();   // the kept list comes from the kernel before this one
+  // Nothing in global memory is written before the wait above: the kernel before this one may belong to an
+  // earlier call on the same workspace and still be running.  The clear is still long before any wait can expire.
+  if (m.clear_status && b == 0 && t0 == 0 && threadIdx.x == 0) *m.status = 0u;
 
   if (warp == 0) {
     // ------------------------------------------------------------ producer: TMA tile + TMA row gathers
@@ -444,6 +446,10 @@ __device__ __forceinline__ void mean_job(const MergeParams& p, int b, int s0, ui
 // follows.  One warp per slot, the whole row in flight at once.
 __global__ void __launch_bounds__(256) pack_kept_norm_kernel(MergeParams m, int rows_packed) {
   grid_dependency_launch();
+  // The kernel before this one may be the persistent kernel of an earlier call on the same workspace, which lets
+  // its successor start early and goes on reading the counters, the packed rows and the norms: every write of
+  // this kernel therefore comes after the wait.  (The kept list also comes from the kernel before this one.)
+  grid_dependency_wait();
   if (blockIdx.x == 0 && blockIdx.y == 0) {
     if (threadIdx.x == 0) *m.status = 0u;
     for (int i = threadIdx.x; i <= m.instances; i += 256) m.counters[i] = 0;
@@ -457,7 +463,6 @@ __global__ void __launch_bounds__(256) pack_kept_norm_kernel(MergeParams m, int 
     for (int v = lane; v < vecs; v += 32) st_16(dst + v, make_uint4(0u, 0u, 0u, 0u));
     return;
   }
-  grid_dependency_wait();   // the kept list comes from the kernel before this one
   const int t = min(max(m.kept[static_cast<size_t>(b) * m.n_kept + s], 0), m.n_tokens - 1);
   const uint4* src = reinterpret_cast<const uint4*>(
       static_cast<const __nv_bfloat16*>(m.metric) + (static_cast<size_t>(b) * m.row_len + m.cls_offset + t) * m.metric_dim);

@@ -54,9 +54,11 @@ vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStre
 
 }  // namespace vscan
 
-using namespace vscan;
+namespace vscan {
 
-static vscan_status validate_score(const vscan_score_desc* d) {
+// Argument checks shared by vscan_score and vscan_score_qk_static.  Shape limits of this build are refused
+// here (VSCAN_ERR_UNSUPPORTED), before anything is enqueued.
+vscan_status validate_score(const vscan_score_desc* d) {
   if (!d || !d->scores) return VSCAN_ERR_INVALID_ARG;
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
   if (!aligned16(d->scores)) return VSCAN_ERR_INVALID_ARG;
@@ -64,8 +66,9 @@ static vscan_status validate_score(const vscan_score_desc* d) {
   if (d->mode == VSCAN_SCORE_ROW) {
     if (!d->attn || !aligned16(d->attn)) return VSCAN_ERR_INVALID_ARG;
     if (d->instances < 0 || d->heads <= 0 || d->n_tokens < 0 || d->cls_offset < 0 ||
-        d->row_len < d->cls_offset + d->n_tokens)
+        static_cast<long long>(d->row_len) < static_cast<long long>(d->cls_offset) + d->n_tokens)
       return VSCAN_ERR_INVALID_ARG;
+    if (d->instances > 65535) return VSCAN_ERR_UNSUPPORTED;
     if (overlaps(d->scores, static_cast<size_t>(d->instances) * d->n_tokens * 4, d->attn,
                  static_cast<size_t>(d->instances) * d->heads * d->row_len * e))
       return VSCAN_ERR_INVALID_ARG;
@@ -75,11 +78,14 @@ static vscan_status validate_score(const vscan_score_desc* d) {
     if (!d->q || !d->k || !aligned16(d->q) || !aligned16(d->k)) return VSCAN_ERR_INVALID_ARG;
     if (d->batch < 0 || d->q_heads <= 0 || d->kv_heads <= 0 || d->q_heads % d->kv_heads ||
         d->seq_len <= 0 || d->head_dim <= 0 || d->span_begin < 0 || d->span_len < 0 ||
-        d->span_begin + d->span_len > d->seq_len)
+        static_cast<long long>(d->span_begin) + d->span_len > static_cast<long long>(d->seq_len))
       return VSCAN_ERR_INVALID_ARG;
     if (d->softmax_span != VSCAN_SPAN_ONLY && d->softmax_span != VSCAN_SPAN_FULL)
       return VSCAN_ERR_INVALID_ARG;
     if (d->head_dim % 8 || d->head_dim > 256) return VSCAN_ERR_INVALID_ARG;
+    if (d->batch > 65535) return VSCAN_ERR_UNSUPPORTED;
+    const int soft_n = d->softmax_span == VSCAN_SPAN_ONLY ? d->span_len : d->seq_len;
+    if (qk_smem_bytes(d->head_dim, soft_n) > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
     if (overlaps(d->scores, static_cast<size_t>(d->batch) * d->span_len * 4, d->k,
                  static_cast<size_t>(d->batch) * d->kv_heads * d->seq_len * d->head_dim * e) ||
         overlaps(d->scores, static_cast<size_t>(d->batch) * d->span_len * 4, d->q,
@@ -89,6 +95,10 @@ static vscan_status validate_score(const vscan_score_desc* d) {
   }
   return VSCAN_ERR_INVALID_ARG;
 }
+
+}  // namespace vscan
+
+using namespace vscan;
 
 extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
   if (!d || d->mode != VSCAN_SCORE_QK || d->batch <= 0 || d->q_heads <= 0 || d->span_len <= 0) return 0;

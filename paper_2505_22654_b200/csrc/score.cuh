@@ -187,7 +187,8 @@ inline size_t qk_smem_bytes(int head_dim, int soft_n) {
   return (static_cast<size_t>(head_dim) + soft_n) * sizeof(float) + 16;
 }
 
-// Host-side launch shared by the entry points.
+// Host-side argument checks and launch shared by the entry points.
+vscan_status validate_score(const vscan_score_desc* d);
 vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStream_t stream);
 
 }  // namespace vscan

@@ -38,7 +38,15 @@ __global__ void __launch_bounds__(256) static_head_mean_kernel(float* __restrict
   if (j >= span_len) return;
   const float* base = g_static_probs + static_cast<size_t>(blockIdx.y) * q_heads * span_len + j;
   float acc = 0.f;
-  for (int h = 0; h < q_heads; ++h) acc += base[static_cast<size_t>(h) * span_len];
+  int h = 0;
+  for (; h + 8 <= q_heads; h += 8) {   // eight independent loads in flight, added in head order
+    float a[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) a[u] = base[static_cast<size_t>(h + u) * span_len];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc += a[u];
+  }
+  for (; h < q_heads; ++h) acc += base[static_cast<size_t>(h) * span_len];
   scores[static_cast<size_t>(blockIdx.y) * span_len + j] = acc / static_cast<float>(q_heads);
 }
 
@@ -51,20 +59,15 @@ extern "C" size_t vscan_score_qk_static_capacity(void) { return kStaticProbFloat
 extern "C" vscan_status vscan_score_qk_static(const vscan_score_desc* d, void* stream_) {
   if (!d || d->mode != VSCAN_SCORE_QK) return VSCAN_ERR_INVALID_ARG;
   if (d->batch == 0) return VSCAN_OK;
-  if (!d->scores || !d->q || !d->k || !aligned16(d->scores) || !aligned16(d->q) || !aligned16(d->k))
-    return VSCAN_ERR_INVALID_ARG;
-  if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
-  if (d->batch < 0 || d->batch > 65535 || d->q_heads <= 0 || d->kv_heads <= 0 || d->q_heads % d->kv_heads ||
-      d->seq_len <= 0 || d->head_dim <= 0 || d->head_dim % 8 || d->head_dim > 256 || d->span_begin < 0 ||
-      d->span_len < 0 || d->span_begin + d->span_len > d->seq_len)
-    return VSCAN_ERR_INVALID_ARG;
-  if (d->softmax_span != VSCAN_SPAN_ONLY && d->softmax_span != VSCAN_SPAN_FULL) return VSCAN_ERR_INVALID_ARG;
+  // the built-in scratch has a fixed size: refuse anything that does not fit, before looking any further
+  if (d->batch > 0 && d->q_heads > 0 && d->span_len > 0 &&
+      static_cast<size_t>(d->batch) * d->q_heads * d->span_len > kStaticProbFloats)
+    return VSCAN_ERR_UNSUPPORTED;
+  vscan_status st = validate_score(d);   // the same checks as vscan_score, output/input overlap included
+  if (st != VSCAN_OK) return st;
   if (d->span_len == 0) return VSCAN_OK;
-  // the built-in scratch has a fixed size: refuse anything that does not fit
-  if (static_cast<size_t>(d->batch) * d->q_heads * d->span_len > kStaticProbFloats) return VSCAN_ERR_UNSUPPORTED;
-
   float* probs = nullptr;
-  vscan_status st = static_scratch(&probs);
+  st = static_scratch(&probs);
   if (st != VSCAN_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   QkParams p;

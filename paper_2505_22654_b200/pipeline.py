@@ -14,7 +14,8 @@ from . import binding as vb
 class VScanReducer:
     def __init__(self, *, dtype, instances, frames, grid_h, grid_w, cls, D, H, win_h, win_w, k_w, k_g,
                  B, n_sys, n_vis, n_txt, Dh, Hq, Hkv, d, k2, pos_planes=1, scale=None,
-                 softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, fused_select=True, device="cuda"):
+                 softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, fused_select=True, overlap_stages=False,
+                 device="cuda"):
         self.dtype = torch.float32 if dtype in ("f32", torch.float32) else torch.bfloat16
         self.instances, self.frames, self.grid_h, self.grid_w, self.cls = instances, frames, grid_h, grid_w, cls
         self.D, self.H, self.win_h, self.win_w, self.k_w, self.k_g = D, H, win_h, win_w, k_w, k_g
@@ -42,7 +43,8 @@ class VScanReducer:
         }
         self.ws_merge = vb.Workspace(64 << 10, dev)
         self.ws_prune = vb.Workspace(64 << 10, dev)
-        self._sized = False
+        self.overlap_stages, self._side = overlap_stages, None
+        self._reserve()
 
     @classmethod
     def from_config(cls_, cfg, **kw):
@@ -62,8 +64,6 @@ class VScanReducer:
             vb.vscan_score_row(attn_l, self.cls, self.N, out=self.scores_l)
             vb.vscan_select_global_local(self.scores_g, self.scores_l, self.frames, self.grid_h, self.grid_w,
                                          self.win_h, self.win_w, self.k_w, self.k_g, out=self.kept_idx)
-        if not self._sized:
-            self._reserve(x)
         vb.vscan_merge(x, self.cls, self.kept_idx, n_tokens=self.N, path=self.merge_path, out=self.merged,
                        workspace=self.ws_merge)
         return self.merged
@@ -73,18 +73,39 @@ class VScanReducer:
                                   self.scale, self.softmax_span, out=self.out2, workspace=self.ws_prune)
 
     def run(self, attn_g, attn_l, x, q_last, k, v, hidden, pos_ids):
-        self.stage1(attn_g, attn_l, x)
-        return self.stage2(q_last, k, v, hidden, pos_ids)
+        if not self.overlap_stages:
+            self.stage1(attn_g, attn_l, x)
+            return self.stage2(q_last, k, v, hidden, pos_ids)
+        # The two stages of one pass have no data in common (Stage 2 reads the LLM's layer-k tensors,
+        # Stage 1 the encoder's), so they are enqueued as two branches that fork from and join back into
+        # the current stream; captured in a CUDA graph they are two parallel branches of the one graph.
+        # Stage 1 (a few hundred long-lived CTAs that leave DRAM half idle) goes to a high-priority stream,
+        # so that its CTAs take SM slots as the thousands of short row-copy CTAs of Stage 2 retire.
+        cur = torch.cuda.current_stream()
+        if self._side is None:
+            self._side = torch.cuda.Stream(device=self.merged.device, priority=-1)
+        self._side.wait_stream(cur)
+        with torch.cuda.stream(self._side):
+            self.stage1(attn_g, attn_l, x)
+        out = self.stage2(q_last, k, v, hidden, pos_ids)
+        cur.wait_stream(self._side)
+        return out
 
-    def _reserve(self, x):
+    def check(self) -> int:
+        """Synchronises the current stream and reads the device status words of both workspaces: 0, or
+        the status a bounded device-side wait left there (binding.ERR_TIMEOUT).  A pass that timed out has
+        unwritten output rows, so callers that time or trust a pass call this after it."""
+        return max(vb.vscan_check(self.ws_merge), vb.vscan_check(self.ws_prune))
+
+    def _reserve(self):
         import ctypes as C
         L = vb.lib()
-        md = vb.MergeDesc(dtype=vb._dtype_code(x), instances=self.instances, n_kept=self.K1, n_tokens=self.N,
+        code = vb.F32 if self.dtype == torch.float32 else vb.BF16
+        md = vb.MergeDesc(dtype=code, instances=self.instances, n_kept=self.K1, n_tokens=self.N,
                           dim=self.D, row_len=self.L, cls_offset=self.cls)
         self.ws_merge.reserve(L.vscan_merge_workspace_bytes(C.byref(md)))
         pd = vb.PruneDesc(batch=self.B, q_heads=self.Hq, n_vis=self.n_vis)
         self.ws_prune.reserve(L.vscan_llm_prune_workspace_bytes(C.byref(pd)))
-        self._sized = True
 
     # ---- end to end: pinned host buffers in, pinned host buffers out
     def run_host(self, host_in: dict, host_out: dict, dev_in: dict):

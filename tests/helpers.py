@@ -74,3 +74,47 @@ def check_merged(got: torch.Tensor, ref: np.ndarray, dtype: str):
         # one rounding of an fp32 mean: within half a bf16 ulp of the exact mean (+ fp32 slack)
         assert np.all(err <= bf16_half_ulp(ref) * 1.02 + 2e-5), float((err - bf16_half_ulp(ref)).max())
     return float(err.max())
+
+
+# ------------------------------------------------------------------ inputs without planted margins
+NEAR_TIE = 1e-4     # a decision whose fp64 margin is below this may fall either way on the GPU
+
+
+def check_topk_unplanted(got, scores, k, candidates=None) -> int:
+    """Exact top-k on scores that were not margin-planted.  `got` (ascending indices) must have exactly k
+    distinct candidates; it may differ from the oracle's set only by tokens whose fp64 score lies within
+    NEAR_TIE of the oracle's k-th largest, everything else must be the oracle's choice.  Returns the
+    number of tokens in which the two sets differ."""
+    s = np.asarray(scores, dtype=np.float64)
+    cand = np.arange(s.shape[0]) if candidates is None else np.asarray(candidates)
+    ref = vo.topk_lowest_index(s, k, cand)
+    got = np.asarray(got, dtype=np.int64)
+    assert got.shape == ref.shape and np.all(np.diff(got) > 0) and np.isin(got, cand).all()
+    diff = np.setxor1d(got, ref)
+    if diff.size:
+        kth = np.sort(s[cand])[::-1][k - 1]
+        assert np.all(np.abs(s[diff] - kth) < NEAR_TIE), (diff, s[diff], kth)
+    return int(diff.size)
+
+
+def check_merge_unplanted(x, cls, kept, merged, assign, counts, dtype) -> int:
+    """Merge results on features that were not margin-planted.  A token's assignment may differ from the
+    oracle's only where the oracle's best and second-best cosine are closer than NEAR_TIE, and then only
+    to a slot whose cosine is within NEAR_TIE of the best; every other assignment is the oracle's.
+    Counts and merged rows are then checked against Eq. 4 evaluated on the assignment the GPU took.
+    Returns the number of assignments that differ."""
+    x64 = np.asarray(x, dtype=np.float64)
+    kept = np.asarray(kept, dtype=np.int64)
+    _, a_ref, _ = vo.merge(x64, cls, kept)
+    a = assign.cpu().numpy().astype(np.int64)
+    np.testing.assert_array_equal(a[kept], np.arange(kept.size))
+    differ = np.nonzero(a != a_ref)[0]
+    if differ.size:
+        cos = vo.cosine_matrix(x64[cls + differ], x64[cls + kept])
+        best = cos.max(axis=1)
+        taken = cos[np.arange(differ.size), a[differ]]
+        assert np.all(best - taken < NEAR_TIE), (differ, best - taken)
+    m_ref, c_ref = vo.mean_merge(x64, cls, kept, a)
+    np.testing.assert_array_equal(counts.cpu().numpy(), c_ref)
+    check_merged(merged, m_ref, dtype)
+    return int(differ.size)

@@ -108,6 +108,34 @@ def test_score_validation_is_host_side(L):
     assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_WORKSPACE       # no workspace given
     d.span_len = 17
     assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG      # span leaves the sequence
+    d.span_begin, d.span_len = 2 ** 31 - 1, 16                                # the sum must not wrap around
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG
+    assert L.vscan_score_qk_static(C.byref(d), None) == vb.ERR_INVALID_ARG
+    d.span_begin = 0
+    d.scores = FAKE + 0x100000                                                # output on top of the keys
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG
+    assert L.vscan_score_qk_static(C.byref(d), None) == vb.ERR_INVALID_ARG    # same checks in the static variant
+    d.scores = FAKE + 0x800000
+
+
+def test_shape_limits_are_refused_before_anything_is_enqueued(L):
+    """Limits of the build come back as UNSUPPORTED from the host-side checks (no stream, no workspace
+    and fake pointers here: a launch or a memset would fail differently)."""
+    d = vb.ScoreDesc(mode=vb.SCORE_ROW, dtype=vb.BF16, attn=FAKE, instances=70000, heads=2, row_len=8,
+                     cls_offset=0, n_tokens=8, scores=FAKE + 0x10000000)
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_UNSUPPORTED      # grid.y limit
+    q = vb.ScoreDesc(mode=vb.SCORE_QK, dtype=vb.BF16, q=FAKE, k=FAKE + 0x100000, batch=70000, q_heads=2,
+                     kv_heads=2, seq_len=16, head_dim=64, span_begin=0, span_len=16, scale=1.0,
+                     scores=FAKE + 0x40000000)
+    assert L.vscan_score(C.byref(q), None, 0, None) == vb.ERR_UNSUPPORTED
+    q.batch, q.seq_len, q.span_len = 1, 70000, 70000                          # softmax row beyond shared memory
+    assert L.vscan_score(C.byref(q), None, 0, None) == vb.ERR_UNSUPPORTED
+    assert L.vscan_score_qk_static(C.byref(q), None) == vb.ERR_UNSUPPORTED
+    m = vb.MergeDesc(dtype=vb.BF16, path=vb.MERGE_AUTO, x=FAKE, kept_idx=FAKE + 0x40000000, instances=1,
+                     row_len=30000, cls_offset=0, n_tokens=30000, dim=8, n_kept=4, merged=FAKE + 0x50000000)
+    assert L.vscan_merge(C.byref(m), None, 0, None) == vb.ERR_UNSUPPORTED      # member list beyond shared memory
+    m.n_tokens = m.row_len = 29054
+    assert L.vscan_merge(C.byref(m), None, 0, None) == vb.ERR_WORKSPACE       # legal: next check is the workspace
 
 
 def test_merge_and_prune_validation_is_host_side(L):
@@ -137,6 +165,23 @@ def test_merge_and_prune_validation_is_host_side(L):
     p.v = None
     p.n_vis, p.k_keep = 20000, 4
     assert L.vscan_llm_prune(C.byref(p), None, 0, None) == vb.ERR_UNSUPPORTED
+
+
+def test_stale_library_is_rebuilt_or_refused(monkeypatch, tmp_path):
+    """A library that does not match the sources on disk is never loaded silently."""
+    assert not _build._stale()                     # the fixture `L` loaded (and, if needed, rebuilt) it
+    stamp = tmp_path / "stamp"
+    stamp.write_text("0" * 64 + "\n")              # a digest of other sources
+    monkeypatch.setattr(_build, "STAMP_PATH", str(stamp))
+    assert _build._stale()
+    monkeypatch.setattr(vb, "_LIB", None)
+    monkeypatch.setattr(_build, "have_nvcc", lambda: False)
+    with pytest.raises(RuntimeError, match="does not match the sources"):
+        vb.lib()
+    calls = []
+    monkeypatch.setattr(_build, "have_nvcc", lambda: True)
+    monkeypatch.setattr(_build, "build", lambda force=False, **k: calls.append(force) or _build.LIB_PATH)
+    assert vb.lib().vscan_version() > 0 and calls == [False]
 
 
 def test_no_cpu_fallback_when_library_missing(monkeypatch, tmp_path):

@@ -9,7 +9,7 @@ from oracle import plant
 from oracle import vscan_oracle as vo
 from synth import CONFIGS, round_to_dtype
 
-from helpers import TOL_SCORE, check_merged, dev, stage1_case, stage2_case
+from helpers import TOL_SCORE, check_merge_unplanted, check_merged, dev, stage1_case, stage2_case
 
 pytestmark = pytest.mark.gpu
 RNG = np.random.default_rng(7)
@@ -218,13 +218,43 @@ def test_merge_interleaved_many_instances(B, N, D, K1):
         assert (ref[1] == out[1]).float().mean() > 0.999
         for r, o in zip(ref, out):
             assert torch.equal(r[same], o[same])
-    for b in (0, B // 2, B - 1):
-        m, a, cn = vo.merge(x[b], 0, kept[b])
-        agree = out[1][b].cpu().numpy() == a      # unplanted inputs: near-ties may differ, the rest must not
-        assert agree.mean() > 0.98
-        if agree.all():
-            np.testing.assert_array_equal(out[2][b].cpu().numpy(), cn)
-            check_merged(out[0][b], m, "bf16")
+    for b in (0, B // 2, B - 1):                  # unplanted inputs: the near-tie rule decides what may differ
+        n_band = check_merge_unplanted(x[b], 0, kept[b], out[0][b], out[1][b], out[2][b], "bf16")
+        assert n_band <= N // 20
+
+
+@pytest.mark.parametrize("K1", [144, 192])
+@pytest.mark.parametrize("path", ["auto", "interleaved"])
+def test_merge_calls_back_to_back_on_one_workspace(K1, path):
+    """Three vscan_merge calls enqueued on one stream and one workspace with nothing between them (no
+    vscan_check, no synchronisation, different inputs and outputs per call).  The kernels of one call are
+    launched so that they may start while the previous kernel drains; a call must not disturb the counters,
+    packed rows or status word an earlier call is still using.  Every result is checked against the oracle."""
+    B, N, D, calls = 40, 576, 1024, 3
+    cfg = small_cfg("bf16", grid_h=1, grid_w=N, win_h=1, win_w=N, k_w=0, k_g=K1, D=D, C=1, B=B, cls=1)
+    rng = np.random.default_rng(K1)
+    xs, kepts = [], []
+    for c in range(calls):
+        x = round_to_dtype(rng.standard_normal((B, N + 1, D)).astype(np.float32), "bf16")
+        kept = np.stack([np.sort(rng.choice(N, K1, replace=False)) for _ in range(B)])
+        plant.plant_merge(cfg, x, kept, seed=c)
+        xs.append(x); kepts.append(kept)
+    xd = [dev(x, "bf16") for x in xs]
+    kd = [dev(k.astype(np.int32)) for k in kepts]
+    outs = [(torch.empty((B, K1, D), dtype=torch.bfloat16, device="cuda"),) for _ in range(calls)]
+    ws = vs.Workspace(64 << 20)
+    code = vs.MERGE_AUTO if path == "auto" else vs.MERGE_INTERLEAVED
+    torch.cuda.synchronize()
+    res = [vs.vscan_merge(xd[c], 1, kd[c], want_assign=True, want_counts=True, workspace=ws, path=code, out=outs[c][0])
+           for c in range(calls)]
+    assert vs.vscan_check(ws) == 0
+    for c in range(calls):
+        merged, assign, counts = res[c]
+        for b in (0, 17, B - 1):
+            m, a, cn = vo.merge(xs[c][b], 1, kepts[c][b])
+            np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
+            np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
+            check_merged(merged[b], m, "bf16")
 
 
 def test_merge_tensor_path_refuses_fp32():

@@ -392,13 +392,30 @@ def test_compaction_matches_index_select_and_keeps_order():
     assert np.all(np.diff(rows) > 0)
 
 
-# ------------------------------------------------------------------ rounding helper
-def test_round_bf16_matches_torch():
-    a = np.concatenate([RNG.standard_normal(5000) * 3, [0.0, 1.0, -1.0, 1.00390625, 1.01171875]])
-    ref = torch.from_numpy(a).to(torch.bfloat16).to(torch.float64).numpy()
-    got = vo.round_bf16(a)
-    # torch rounds f64 -> bf16 directly; agreement must be exact
-    np.testing.assert_array_equal(got, ref)
+# ------------------------------------------------------------------ helpers the parity tests lean on
+def test_mean_merge_hand_example_and_agreement_with_merge():
+    # five tokens in one dimension, tokens 1 and 3 kept; groups decided by hand: {1, 0, 2} and {3, 4}
+    x = np.array([[2.0], [4.0], [9.0], [10.0], [30.0]])
+    merged, counts = vo.mean_merge(x, 0, np.array([1, 3]), np.array([0, 0, 0, 1, 1]))
+    assert merged[:, 0].tolist() == [(4.0 + 2.0 + 9.0) / 3, (10.0 + 30.0) / 2] and counts.tolist() == [3, 2]
+    # a [CLS] row in front shifts the rows, not the token numbering
+    xc = np.concatenate([[[1000.0]], x])
+    assert np.array_equal(vo.mean_merge(xc, 1, np.array([1, 3]), np.array([0, 0, 0, 1, 1]))[0], merged)
+    # merge() = cosine arg-max followed by exactly this function
+    xr = RNG.standard_normal((41, 12))
+    kept = np.array([3, 8, 20, 33])
+    m, a, c = vo.merge(xr, 1, kept)
+    m2, c2 = vo.mean_merge(xr, 1, kept, a)
+    assert np.array_equal(m, m2) and np.array_equal(c, c2)
+
+
+def test_topk_boundary_gap_hand_values():
+    s = np.array([0.5, 0.1, 0.9, 0.4, 0.7])
+    assert vo.topk_boundary_gap(s, 2) == pytest.approx(0.7 - 0.5)
+    assert vo.topk_boundary_gap(s, 4) == pytest.approx(0.4 - 0.1)
+    assert vo.topk_boundary_gap(s, 1, np.array([1, 3, 4])) == pytest.approx(0.7 - 0.4)   # candidates only
+    assert vo.topk_boundary_gap(s, 0) == float("inf") and vo.topk_boundary_gap(s, 5) == float("inf")
+    assert vo.topk_boundary_gap(np.array([1.0, 1.0, 0.0]), 1) == 0.0                     # an exact tie at the cut
 
 
 # ------------------------------------------------------------------ planted mistakes are caught

@@ -1,10 +1,10 @@
 """vscan_score_qk_static: the entry point for callers that cannot allocate device memory.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already been
-through every other test.  The check is against the library's own workspace-based entry point on the
-same inputs: both run the same arithmetic, so the scores must agree within the score tolerance used
-everywhere else, on two calls in a row (the second one finds the first one's leftovers in the
-built-in scratch and must not be disturbed by them).
+through every other test.  The scores are checked twice over: against the library's own workspace-based
+entry point on the same inputs (same arithmetic, so they must agree within the score tolerance used
+everywhere else) and against the CPU oracle's Eq. 5, on two calls in a row (the second one finds the
+first one's leftovers in the built-in scratch and must not be disturbed by them).
 """
 import ctypes as C
 
@@ -14,6 +14,8 @@ import torch
 
 import paper_2505_22654_b200 as vs
 from paper_2505_22654_b200 import binding as vb
+
+from oracle import vscan_oracle as vo
 
 from helpers import TOL_SCORE
 
@@ -25,6 +27,11 @@ def _inputs(seed, B, Hq, Hkv, S, d, dtype):
     q = torch.randn((B, Hq, d), generator=g).to(dtype).cuda()
     k = torch.randn((B, Hkv, S, d), generator=g).to(dtype).cuda()
     return q, k
+
+
+def _oracle(q, k, b0, n, scale, span=vo.SPAN_ONLY):
+    qn, kn = q.float().cpu().numpy(), k.float().cpu().numpy()
+    return np.stack([vo.score_qk(qn[b], kn[b], b0, n, scale, span) for b in range(qn.shape[0])])
 
 
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
@@ -45,6 +52,9 @@ def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
     assert float((got1 - ref1).abs().max()) <= TOL_SCORE
     assert float((got2 - ref2).abs().max()) <= TOL_SCORE
     np.testing.assert_allclose(got1.sum(-1).cpu().numpy(), 1.0, atol=1e-5)
+    # the same two results against the CPU oracle (Eq. 5 in float64 on the same rounded inputs)
+    assert np.abs(got1.cpu().numpy() - _oracle(q, k, 35, 320, 128 ** -0.5)).max() <= TOL_SCORE
+    assert np.abs(got2.cpu().numpy() - _oracle(q2, k2, 7, 257, 0.125, vo.SPAN_FULL)).max() <= TOL_SCORE
     # and the first shape once more gives the first answer again
     got3 = vs.vscan_score_qk_static(q, k, 35, 320, 128 ** -0.5, out3)
     assert float((got3 - ref1).abs().max()) <= TOL_SCORE
