@@ -26,7 +26,7 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-from synth import CONFIGS, stage1_inputs, stage2_inputs, sweep_config  # noqa: E402
+from synth import CONFIGS, schedule_points, stage1_inputs, stage2_inputs, sweep_config  # noqa: E402
 
 METRIC = "VScan reduction images/s (Stage1+Stage2) at 2880 visual tokens"
 UNIT = "images/s"
@@ -36,20 +36,24 @@ MERGE_KERNELS = ("kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", 
 
 # ------------------------------------------------------------------ algorithmic work per step
 def algorithmic_bytes(cfg) -> dict:
-    """Bytes each call has to move per step (whole batch): inputs read once, outputs written once."""
+    """Bytes each call has to move per step (whole batch): every input byte read once, every output
+    byte written once.  The K rows of the Stage-2 survivors are read by the scoring (the whole visual
+    span of K) and are not charged a second time to the compaction."""
     e, I, B = cfg.elem_bytes, cfg.instances, cfg.B
+    k_survivors = B * cfg.Hkv * cfg.k2 * cfg.d * e          # part of the span the scoring already read
     row = {
-        "row_mean": I * (cfg.H * cfg.L * e + cfg.N * 4),                       # one launch (two per step)
-        "select": I * (2 * cfg.N * 4 + cfg.K1 * 4),
+        "row_mean": I * (cfg.H * cfg.L * e + cfg.N * 4),                       # un-fused ROW-mode score
+        "select": I * (2 * cfg.N * 4 + cfg.K1 * 4),                            # un-fused selection
+        "score_select": 2 * I * cfg.H * cfg.L * e + I * (2 * cfg.N * 4 + cfg.K1 * 4),   # Eq. 2 + Eq. 3 fused
         "merge": I * (cfg.N * cfg.D * e + cfg.K1 * 4 + cfg.K1 * cfg.D * e),     # X once + merged out
         "qk_softmax": B * (cfg.Hkv * cfg.n_vis * cfg.d * e + cfg.Hq * cfg.d * e),
         "prune_topk": B * cfg.k2 * 4,
-        "compact": B * 2 * cfg.S_out * (cfg.Dh * e + 2 * cfg.Hkv * cfg.d * e + cfg.pos_planes * 4),
+        "compact": B * 2 * cfg.S_out * (cfg.Dh * e + 2 * cfg.Hkv * cfg.d * e + cfg.pos_planes * 4) - k_survivors,
     }
-    row["score_select"] = 2 * I * cfg.H * cfg.L * e + I * (2 * cfg.N * 4 + cfg.K1 * 4)   # fused Eq. 2 + Eq. 3
     row["prune_fused"] = row["qk_softmax"] + row["prune_topk"] + row["compact"]   # Stage 2 in one launch
-    row["step"] = 2 * row["row_mean"] + row["select"] + row["merge"] + row["qk_softmax"] + \
-        row["prune_topk"] + row["compact"]
+    # the step as it is launched: fused score + select, the merge call, Stage 2
+    row["step"] = row["score_select"] + row["merge"] + row["prune_fused"]
+    row["stage2_only"] = row["prune_fused"]
     return row
 
 
@@ -241,7 +245,7 @@ def build_sets(cfg, n_sets: int, device):
     return sets
 
 
-def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=True):
+def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=True, run_stage1=True):
     """Times one workload on this rank's GPU; rank 0 gets the JSON-able result dict, others None."""
     import torch
 
@@ -254,7 +258,8 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
     warmup = max(args.warmup, 3)
     sets = build_sets(cfg, n_sets, device)
     reducers = [vs.VScanReducer.from_config(cfg, device=device, merge_path=args.merge_path,
-                                            overlap_stages=args.overlap_stages) for _ in range(n_sets)]
+                                            overlap_stages=args.overlap_stages, run_stage1=run_stage1)
+                for _ in range(n_sets)]
     stream = torch.cuda.Stream(device)
     launches_per_step = 0
     with torch.cuda.stream(stream):
@@ -299,6 +304,8 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
         if dist is not None:
             dist.barrier()
         ms_total = max_over_ranks(ev0.elapsed_time(ev1), dist, device)
+        # a bounded device-side wait that ran out leaves unwritten rows behind: such a run is not a measurement
+        status = max(r.check() for r in reducers)
 
         # ---- per-kernel durations: the same steps launched directly, each kernel between two events
         prof_steps = max(1, min(args.steps, 30))
@@ -339,6 +346,8 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
     if rank == 0:
         peak, peak_kind = measured_peaks()
         alg = algorithmic_bytes(cfg)
+        if not run_stage1:
+            alg["step"] = alg["stage2_only"]
         ms_step = ms_total / args.steps
         kernels = {}
         total_k = sum(sum(v) for v in per_kernel.values())
@@ -379,6 +388,7 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
                       "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names),
                       "assign_kernel": next((n for n in ("merge_persistent", "assign_tensor", "assign_simt", "merge_fused") if n in kernels), None)},
             "gpu_launches": launches_per_step * args.steps,
+            "status": status,
             "clocks": clocks,
             "e2e": e2e,
             "cpu_baseline": cpu,
@@ -422,17 +432,23 @@ def run_sweep(args, rank, world, local_rank, dist):
     points += [("sweep b=%d %s" % (b, r), sweep_config(b, r), 0) for r in SWEEP_BUDGETS for b in SWEEP_BATCHES]
     points += [("simt b=32 %s" % r, sweep_config(32, r), 1) for r in SWEEP_BUDGETS]
     points += [("tensor b=32 %s" % r, sweep_config(32, r), 2) for r in SWEEP_BUDGETS]
-    for label, cfg, path in points:
+    points = [(label, cfg, path, True) for label, cfg, path in points]
+    # the paper's pruning schedules as throughput points (Table 1, Table 6(a)/(b), App. B.1)
+    points += [(label, cfg, 0, s1) for label, cfg, s1 in schedule_points()]
+    if args.sweep_filter:
+        points = [p for p in points if args.sweep_filter in p[0]]
+    for label, cfg, path, s1 in points:
         args.merge_path = path
         steps = args.steps
         args.steps = max(10, min(steps, int(2e5 / max(cfg.B, 1)) // 10 * 10)) if cfg.B > 64 else steps
-        line = measure(args, cfg, rank, world, local_rank, dist, with_e2e=False, with_cpu=False)
+        line = measure(args, cfg, rank, world, local_rank, dist, with_e2e=False, with_cpu=False, run_stage1=s1)
         args.steps = steps
         if rank != 0:
             continue
         k = line["kernels"]
         assign = line["merge"]["assign_kernel"]
-        out = {"point": label, "workload": cfg.name, "B": cfg.B, "K1": cfg.K1, "dtype": cfg.dtype,
+        out = {"point": label, "workload": cfg.name, "B": cfg.B, "K1": cfg.K1, "n_vis": cfg.n_vis, "k2": cfg.k2,
+               "dtype": cfg.dtype, "status": line["status"],
                "images_per_s": round(line["value"], 1), "ms_per_step": round(line["ms_per_step"], 4),
                "hbm_frac": round(line["step_hbm"]["frac"], 3), "merge_us": round(line["merge"]["us"], 1),
                "assign_kernel": assign, "assign_us": round(k[assign]["avg_us"], 1) if assign else None,
@@ -454,7 +470,9 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--overlap-stages", action="store_true", help="Stage 1 and Stage 2 as two parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", action="store_true", help="all named workloads and the batch x retention sweep")
+    ap.add_argument("--sweep", action="store_true",
+                    help="all named workloads, the batch x retention sweep and the paper's pruning schedules")
+    ap.add_argument("--sweep-filter", default="", help="with --sweep: only the points whose label contains this")
     args = ap.parse_args()
     if args.workload.startswith("sweep:"):
         _, b, r = args.workload.split(":")

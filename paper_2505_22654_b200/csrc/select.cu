@@ -18,6 +18,8 @@ struct SelectParams {
   int32_t* kept_idx;
   uint8_t* kept_mask;
   int n, frames, grid_h, grid_w, win_h, win_w, k_w, k_g, windows, wins_per_row, wins_per_frame;
+  // ceil(2^32 / d) for d = tokens per frame, grid_w, win_h, win_w: umulhi(x, rcp) == x / d for x * d < 2^32
+  uint32_t rcp_frame, rcp_grid_w, rcp_win_h, rcp_win_w;
 };
 
 // Head mean of one token's attention entries, heads ascending (same arithmetic as the ROW-mode score).
@@ -148,6 +150,183 @@ __global__ void __launch_bounds__(1024) select_kernel(SelectParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Instances of at most 1024 tokens: one thread per token, keys in registers.
+//   loads   fused form: the instance's [heads][row_len] block of each attention tensor is one contiguous run
+//           of memory; when it is 16-byte aligned it comes in as one bulk copy per tensor (mbarrier with
+//           transaction count) and the head means are taken out of shared memory, else (or if the copy does
+//           not arrive within the wait's bound) with one strided load per head as in the large kernel
+//   local   one warp per window, rank counting in registers (or the 32-step bit select for windows above 64)
+//   global  the k_g-th largest key of the complement by binary search on the key's bits, one
+//           barrier-with-count per varying bit (bits that all candidates share are skipped)
+//   union   warp ballots and one exchange of per-warp counts: position = kept tokens before mine
+// dynamic shared memory: keys_l[n] | taken[n] bytes (padded to 16) | staging for the two attention blocks
+// x / d through the host's ceil(2^32 / d) (d = 1 has no 32-bit reciprocal)
+__device__ __forceinline__ int quot(int x, int d, uint32_t rcp) {
+  return d == 1 ? x : static_cast<int>(__umulhi(static_cast<uint32_t>(x), rcp));
+}
+
+struct SmallScratch {
+  int warp_sure[32], warp_eq[32];
+  uint32_t bits_or, bits_and;
+  unsigned long long mbar;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(1024) select_small_kernel(SelectParams p, int stage_bytes) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  uint32_t* keys_l = reinterpret_cast<uint32_t*>(smem_raw);
+  uint8_t* taken = reinterpret_cast<uint8_t*>(keys_l + p.n);
+  __shared__ SmallScratch sc;
+  grid_dependency_launch();
+
+  const int b = blockIdx.x, i = threadIdx.x, lane = i & 31, warp = i >> 5, nwarps = blockDim.x >> 5;
+  const bool live = i < p.n;
+  float g = 0.f, l = 0.f;
+  if constexpr (std::is_void<T>::value) {
+    if (live) {
+      g = p.scores_global[static_cast<size_t>(b) * p.n + i];
+      l = p.scores_local[static_cast<size_t>(b) * p.n + i];
+    }
+  } else {
+    const size_t block_elems = static_cast<size_t>(p.heads) * p.row_len;
+    const T* ag = static_cast<const T*>(p.attn_global) + static_cast<size_t>(b) * block_elems;
+    const T* al = static_cast<const T*>(p.attn_local) + static_cast<size_t>(b) * block_elems;
+    const bool same = p.attn_local == p.attn_global;
+    bool staged = false;
+    if (stage_bytes > 0) {
+      unsigned char* stage = smem_raw + ((static_cast<size_t>(p.n) * 5 + 15) / 16) * 16;
+      const uint32_t bar = static_cast<uint32_t>(__cvta_generic_to_shared(&sc.mbar));
+      if (i == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(same ? stage_bytes : 2 * stage_bytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(stage))), "l"(ag), "r"(stage_bytes), "r"(bar) : "memory");
+        if (!same)
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                       ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(stage + stage_bytes))), "l"(al), "r"(stage_bytes), "r"(bar) : "memory");
+      }
+      __syncthreads();   // the barrier is initialised before anyone polls it
+      uint32_t done = 0;
+      for (uint32_t spin = 0; spin < (1u << 20) && !done; ++spin)
+        asm volatile("{\n\t.reg .pred q;\n\tmbarrier.try_wait.parity.shared::cta.b64 q, [%1], 0;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                     : "=r"(done) : "r"(bar) : "memory");
+      staged = __syncthreads_and(done != 0) != 0;   // all or nobody: a copy that did not arrive is not relied on
+      if (staged && live) {
+        const T* sg = reinterpret_cast<const T*>(stage) + p.cls_offset + i;
+        const T* sl = same ? sg : reinterpret_cast<const T*>(stage + stage_bytes) + p.cls_offset + i;
+        for (int h = 0; h < p.heads; ++h) g += to_float(sg[static_cast<size_t>(h) * p.row_len]);
+        g /= static_cast<float>(p.heads);
+        if (same) l = g;
+        else {
+          for (int h = 0; h < p.heads; ++h) l += to_float(sl[static_cast<size_t>(h) * p.row_len]);
+          l /= static_cast<float>(p.heads);
+        }
+      }
+    }
+    if (!staged && live) {
+      g = head_mean_of(ag + p.cls_offset + i, p.heads, p.row_len);
+      l = same ? g : head_mean_of(al + p.cls_offset + i, p.heads, p.row_len);
+    }
+    if (live) {
+      if (p.scores_global_out) p.scores_global_out[static_cast<size_t>(b) * p.n + i] = g;
+      if (p.scores_local_out) p.scores_local_out[static_cast<size_t>(b) * p.n + i] = l;
+    }
+  }
+  const uint32_t key = float_to_key(g);
+  if (live) { keys_l[i] = float_to_key(l); taken[i] = 0; }
+  if (i == 0) { sc.bits_or = 0u; sc.bits_and = 0xFFFFFFFFu; }
+  __syncthreads();
+
+  // ---- local scan.  Windows of up to 128 tokens: every thread ranks its own token among the tokens of its
+  // window (kept iff fewer than k_w of them beat it: larger key, or equal key and lower index), all warps busy
+  // and no warp-wide chain.  Larger windows: one warp per window with the 32-step bit select.
+  bool mine_taken = false;
+  if (p.k_w > 0) {
+    const int m = p.win_h * p.win_w;
+    if (m <= 128) {
+      if (live) {
+        // quotients by multiplication with the host's rounded-up reciprocals (exact for these ranges)
+        const int per_frame = p.grid_h * p.grid_w;
+        const int f = quot(i, per_frame, p.rcp_frame), rem = i - f * per_frame;
+        const int r = quot(rem, p.grid_w, p.rcp_grid_w), c = rem - r * p.grid_w;
+        const int wr = quot(r, p.win_h, p.rcp_win_h), wc = quot(c, p.win_w, p.rcp_win_w);
+        const int base = f * per_frame + wr * p.win_h * p.grid_w + wc * p.win_w;
+        const uint32_t mykey = keys_l[i];
+        int rank = 0;
+        for (int wy = 0; wy < p.win_h; ++wy) {
+          const int row = base + wy * p.grid_w;
+          for (int wx0 = 0; wx0 < p.win_w; wx0 += 8) {     // eight independent loads per round
+            uint32_t kt[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) kt[u] = wx0 + u < p.win_w ? keys_l[row + wx0 + u] : 0u;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const int t = row + wx0 + u;
+              rank += (wx0 + u < p.win_w) && ((kt[u] > mykey) || (kt[u] == mykey && t < i));
+            }
+          }
+        }
+        mine_taken = rank < p.k_w;
+      }
+    } else {
+      for (int w = warp; w < p.windows; w += nwarps) {
+        const int f = w / p.wins_per_frame, wr = (w % p.wins_per_frame) / p.wins_per_row, wc = w % p.wins_per_row;
+        const int base = f * p.grid_h * p.grid_w + wr * p.win_h * p.grid_w + wc * p.win_w;
+        const int win_w = p.win_w, grid_w = p.grid_w;
+        auto token_of = [=](int q) { return base + (q / win_w) * grid_w + (q % win_w); };
+        warp_select_mark(keys_l, m, p.k_w, token_of, taken);
+      }
+      __syncthreads();
+      mine_taken = live && taken[i];
+    }
+  }
+  const bool cand = live && !mine_taken;
+
+  // ---- global scan: threshold = k_g-th largest candidate key, need = how many keys equal to it belong to the set
+  uint32_t thr = 0;
+  int need = 0;
+  if (p.k_g > 0) {
+    // bits on which all candidates agree cannot decide anything: start below them
+    const uint32_t wo = __reduce_or_sync(0xffffffffu, cand ? key : 0u);
+    const uint32_t wa = __reduce_and_sync(0xffffffffu, cand ? key : 0xFFFFFFFFu);
+    if (lane == 0) { atomicOr(&sc.bits_or, wo); atomicAnd(&sc.bits_and, wa); }
+    __syncthreads();
+    const uint32_t differ = sc.bits_or ^ sc.bits_and;
+    const int top = differ ? 31 - __clz(differ) : -1;            // highest bit that varies
+    // the leading bits all candidates share (all 32 when no bit varies: the threshold is that one key)
+    thr = top < 0 ? sc.bits_and : (top == 31 ? 0u : (sc.bits_and & ~((2u << top) - 1u)));
+    for (int bit = top; bit >= 0; --bit) {
+      const uint32_t t = thr | (1u << bit);
+      if (__syncthreads_count(cand && key >= t) >= p.k_g) thr = t;
+    }
+    need = p.k_g - __syncthreads_count(cand && key > thr);
+  }
+
+  // ---- union, ascending: a token's position is the number of kept tokens before it
+  const bool sure = mine_taken || (cand && p.k_g > 0 && key > thr);
+  const bool eq = cand && p.k_g > 0 && key == thr;
+  const unsigned b_sure = __ballot_sync(0xffffffffu, sure), b_eq = __ballot_sync(0xffffffffu, eq);
+  if (lane == 0) { sc.warp_sure[warp] = __popc(b_sure); sc.warp_eq[warp] = __popc(b_eq); }
+  __syncthreads();
+  int ws = lane < nwarps ? sc.warp_sure[lane] : 0, we = lane < nwarps ? sc.warp_eq[lane] : 0;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int a = __shfl_up_sync(0xffffffffu, ws, o), c = __shfl_up_sync(0xffffffffu, we, o);
+    if (lane >= o) { ws += a; we += c; }
+  }
+  const int sure_warps = warp > 0 ? __shfl_sync(0xffffffffu, ws, warp - 1) : 0;   // inclusive sums of the warps before mine
+  const int eq_warps = warp > 0 ? __shfl_sync(0xffffffffu, we, warp - 1) : 0;
+  const unsigned lt = (1u << lane) - 1u;
+  const int eq_rank = eq_warps + __popc(b_eq & lt);                 // equal keys before mine, in index order
+  const bool keep = sure || (eq && eq_rank < need);
+  const int pos = sure_warps + __popc(b_sure & lt) + min(eq_rank, need);
+  const int k1 = p.windows * p.k_w + p.k_g;
+  if (keep && pos < k1) p.kept_idx[static_cast<size_t>(b) * k1 + pos] = i;
+  if (p.kept_mask && live) p.kept_mask[static_cast<size_t>(b) * p.n + i] = keep ? 1 : 0;
+}
+
 }  // namespace vscan
 
 using namespace vscan;
@@ -177,6 +356,9 @@ static void fill_params(SelectParams& p, const vscan_select_desc* d, long long n
   p.win_h = d->win_h; p.win_w = d->win_w; p.k_w = d->k_per_window; p.k_g = d->k_global;
   p.windows = windows; p.wins_per_row = d->grid_w / d->win_w;
   p.wins_per_frame = (d->grid_h / d->win_h) * p.wins_per_row;
+  auto rcp = [](long long v) { return v <= 1 ? 0u : static_cast<uint32_t>(((1ull << 32) + v - 1) / v); };
+  p.rcp_frame = rcp(1ll * d->grid_h * d->grid_w); p.rcp_grid_w = rcp(d->grid_w);
+  p.rcp_win_h = rcp(d->win_h); p.rcp_win_w = rcp(d->win_w);
 }
 
 // One warp per window while there are enough windows to fill the block.
@@ -185,6 +367,23 @@ static int select_threads(long long n, int windows) {
   // a thread per token where that is possible, so that the scores of an instance are read in one round of loads
   if (n > 512 && n <= 1024) return static_cast<int>((n + 31) / 32 * 32);
   return windows > 8 || n > 256 ? 512 : 256;
+}
+
+// ---- the one-thread-per-token kernel
+constexpr long long kSmallSelect = 1024;
+static int small_threads(long long n) { return static_cast<int>((n + 31) / 32 * 32); }
+// keys_l + taken flags, then (fused form) the staged attention blocks
+static size_t small_smem(long long n, size_t stage_bytes, bool two) {
+  return (static_cast<size_t>(n) * 5 + 15) / 16 * 16 + stage_bytes * (two ? 2 : 1);
+}
+// Bytes of one instance's [heads][row_len] block when it can come in as one bulk copy: every block starts on a
+// 16-byte boundary, its size is a multiple of 16 bytes, and both blocks fit beside the keys.  Else 0.
+static size_t stage_block_bytes(const vscan_score_select_desc* d, long long n) {
+  const size_t bytes = static_cast<size_t>(d->heads) * d->row_len * dtype_bytes(d->dtype);
+  if (bytes % 16 != 0 || bytes >= (1u << 20)) return 0;
+  const bool two = d->attn_global != d->attn_local;
+  if (small_smem(n, bytes, two) > 160 * 1024) return 0;
+  return bytes;
 }
 
 extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
@@ -206,9 +405,13 @@ extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, vo
 
   SelectParams p;
   fill_params(p, d, n, windows);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n <= kSmallSelect) {
+    VSCAN_LAUNCH("select", st, select_small_kernel<void><<<d->instances, small_threads(n), small_smem(n, 0, false), st>>>(p, 0));
+    return VSCAN_OK;
+  }
   const size_t smem = static_cast<size_t>(n) * 9 + 16;
   VSCAN_CUDA_TRY(allow_smem(select_kernel<void>, smem));
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
   VSCAN_LAUNCH("select", st, select_kernel<void><<<d->instances, select_threads(n, windows), smem, st>>>(p));
   return VSCAN_OK;
 }
@@ -246,8 +449,20 @@ extern "C" vscan_status vscan_score_select(const vscan_score_select_desc* d, voi
   p.scores_global_out = const_cast<float*>(sd->scores_global);
   p.scores_local_out = const_cast<float*>(sd->scores_local);
   p.heads = d->heads; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
-  const size_t smem = static_cast<size_t>(n) * 9 + 16;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (n <= kSmallSelect) {
+    const size_t stage = stage_block_bytes(d, n);
+    const size_t sm = small_smem(n, stage, d->attn_global != d->attn_local);
+    if (d->dtype == VSCAN_F32) {
+      VSCAN_CUDA_TRY(allow_smem(select_small_kernel<float>, sm));
+      VSCAN_LAUNCH("score_select", st, select_small_kernel<float><<<sd->instances, small_threads(n), sm, st>>>(p, static_cast<int>(stage)));
+    } else {
+      VSCAN_CUDA_TRY(allow_smem(select_small_kernel<__nv_bfloat16>, sm));
+      VSCAN_LAUNCH("score_select", st, select_small_kernel<__nv_bfloat16><<<sd->instances, small_threads(n), sm, st>>>(p, static_cast<int>(stage)));
+    }
+    return VSCAN_OK;
+  }
+  const size_t smem = static_cast<size_t>(n) * 9 + 16;
   const int threads = select_threads(n, windows);
   if (d->dtype == VSCAN_F32) {
     VSCAN_CUDA_TRY(allow_smem(select_kernel<float>, smem));

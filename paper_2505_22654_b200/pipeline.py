@@ -15,7 +15,7 @@ class VScanReducer:
     def __init__(self, *, dtype, instances, frames, grid_h, grid_w, cls, D, H, win_h, win_w, k_w, k_g,
                  B, n_sys, n_vis, n_txt, Dh, Hq, Hkv, d, k2, pos_planes=1, scale=None,
                  softmax_span=vb.SPAN_ONLY, merge_path=vb.MERGE_AUTO, fused_select=True, overlap_stages=False,
-                 device="cuda"):
+                 run_stage1=True, device="cuda"):
         self.dtype = torch.float32 if dtype in ("f32", torch.float32) else torch.bfloat16
         self.instances, self.frames, self.grid_h, self.grid_w, self.cls = instances, frames, grid_h, grid_w, cls
         self.D, self.H, self.win_h, self.win_w, self.k_w, self.k_g = D, H, win_h, win_w, k_w, k_g
@@ -43,7 +43,7 @@ class VScanReducer:
         }
         self.ws_merge = vb.Workspace(64 << 10, dev)
         self.ws_prune = vb.Workspace(64 << 10, dev)
-        self.overlap_stages, self._side = overlap_stages, None
+        self.overlap_stages, self._side, self.run_stage1 = overlap_stages, None, run_stage1
         self._reserve()
 
     @classmethod
@@ -73,6 +73,8 @@ class VScanReducer:
                                   self.scale, self.softmax_span, out=self.out2, workspace=self.ws_prune)
 
     def run(self, attn_g, attn_l, x, q_last, k, v, hidden, pos_ids):
+        if not self.run_stage1:      # schedules that prune inside the LLM only
+            return self.stage2(q_last, k, v, hidden, pos_ids)
         if not self.overlap_stages:
             self.stage1(attn_g, attn_l, x)
             return self.stage2(q_last, k, v, hidden, pos_ids)

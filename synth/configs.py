@@ -36,6 +36,7 @@ class VScanConfig:
     d: int                  # head dim
     k2: int                 # Stage-2 survivors per image
     pos_planes: int = 1     # 1, or 3 for three-plane rotary position ids
+    vis_in: int = 0         # visual tokens entering Stage 2 when that is not C * K1 (schedules without Stage 1)
 
     @property
     def N(self) -> int:
@@ -59,7 +60,7 @@ class VScanConfig:
 
     @property
     def n_vis(self) -> int:
-        return self.C * self.K1
+        return self.vis_in if self.vis_in > 0 else self.C * self.K1
 
     @property
     def S(self) -> int:
@@ -105,6 +106,48 @@ def sweep_config(batch: int, retention: str) -> VScanConfig:
     k1 = k_g + base.W * k_w
     return base.with_(name=f"sweep_b{batch}_{retention}", config_id=4, B=batch, k_w=k_w, k_g=k_g,
                       k2=(base.C * k1) // 2)
+
+
+def _split_budget(base: VScanConfig, kept: int, local_share: float):
+    """(k_w, k_g) for `kept` tokens per crop with `local_share` of them from the local scan: the per-window
+    budget is the share divided evenly over the windows, rounded down; the global scan takes the rest, so
+    the total is exact (the rule of the 25 % sweep point above)."""
+    k_w = min(int(kept * local_share) // base.W, base.win_h * base.win_w)
+    return k_w, kept - base.W * k_w
+
+
+# (pruning layer k, R2 in percent) as printed in Table 1
+TABLE1_SETTINGS = ((2, 73.3), (8, 66.7), (12, 60.0), (16, 50.0), (20, 33.3), (24, 0.0))
+
+
+def schedule_points():
+    """Pruning schedules of the paper as throughput workloads at the 2880-token shape (5 crops of 576
+    patches, batch 32).  Only counts change; the layer index of a schedule does not change the work.
+    -> list of (label, config, runs_stage1).
+      Table 1: global scan only to R1 = 50 % / 25 %, then the (pruning layer k, R2) pairs the table prints
+               (each pair averages 75 % of the Stage-1 set over the 32 LLM layers).
+      Table 6(a): R1 / R2 pairs with the same 11.1 % average; Table 6(b): global:local share at R1 = 16.7 %.
+      App. B.1: a schedule without Stage 1 that prunes all 2880 tokens to 5.2 % at an early layer."""
+    base = CONFIGS[2]
+    pts = []
+    for r1, kept in (("50%", 288), ("25%", 144)):
+        for k, r2 in TABLE1_SETTINGS:
+            k2 = round(base.C * kept * r2 / 100)
+            pts.append((f"table1 R1={r1} k={k}", base.with_(name=f"table1_{kept}_k{k}", config_id=5, k_w=0, k_g=kept,
+                                                             k2=k2), True))
+    for r1, kept, r2 in (("11.1%", 64, 1.0), ("13.3%", 77, 2 / 3), ("14.8%", 85, 0.5), ("16.7%", 96, 1 / 3),
+                         ("22.2%", 128, 0.0)):
+        k_w, k_g = _split_budget(base, kept, 0.5)
+        pts.append((f"table6a R1={r1} R2={100 * r2:.1f}%", base.with_(name=f"table6a_{kept}", config_id=6, k_w=k_w,
+                                                                      k_g=k_g, k2=round(base.C * kept * r2)), True))
+    for share in (1.0, 0.75, 0.5, 0.25, 0.0):
+        k_w, k_g = _split_budget(base, 96, share)
+        pts.append((f"table6b global:local={100 - 100 * share:.0f}:{100 * share:.0f}",
+                    base.with_(name=f"table6b_{int(100 * share)}", config_id=7, k_w=k_w, k_g=k_g, k2=base.C * 32), True))
+    full = base.C * base.N
+    pts.append(("appB1 no stage 1, 5.2% from an early layer",
+                base.with_(name="appB1_5.2", config_id=8, vis_in=full, k2=round(0.052 * full)), False))
+    return pts
 
 
 def tiny_config(dtype: str = "f32", **kw) -> VScanConfig:

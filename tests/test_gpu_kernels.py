@@ -308,6 +308,14 @@ def test_cls_scores_from_q_and_k_eq1_eq2(dtype):
     g32 = got.cpu().numpy()
     for b in range(B):
         np.testing.assert_array_equal(kept[b], vo.select_global_local(g32[b], g32[b], 1, 24, 24, 6, 6, 2, 32)[0])
+    # The other reading of Eq. 1 (K_V = the patch keys only, [CLS] left out of the softmax) is the same
+    # call with SPAN_ONLY: each head's row is the full-softmax row renormalised over the patches.
+    alt = vs.vscan_score_qk(dev(q, dtype), dev(k, dtype), 1, N, scale, vs.SPAN_ONLY).cpu().numpy()
+    for b in range(B):
+        rows = vo.cls_attention_rows(q[b], k[b], scale)[:, 1:]
+        ref_alt = (rows / rows.sum(axis=1, keepdims=True)).mean(axis=0)
+        assert np.abs(alt[b] - ref_alt).max() <= TOL_SCORE
+        assert abs(alt[b].sum() - 1.0) < 1e-5
 
 
 # ------------------------------------------------------------------ vscan_llm_prune
@@ -353,6 +361,47 @@ def test_multi_turn_reselection_from_the_same_pool():
             np.testing.assert_array_equal(out["hidden"][b].float().cpu().numpy(), base["hidden"][b][rows])
         kept_turns.append(out["kept_vis"].cpu().numpy().copy())
     assert any(not np.array_equal(kept_turns[0], k) for k in kept_turns[1:])     # different questions, different sets
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_prune_schedule_over_several_layers(dtype):
+    """Stage 2 applied at three LLM layers in a row on the shrinking sequence (the multi-layer schedules
+    App. B.1 compares with): each layer brings its own q / K / V for the current sequence, while hidden
+    states and position ids are the previous call's output.  Every call is checked against the oracle run
+    on the oracle's previous output, bit for bit, and the position ids end up naming the original tokens."""
+    cfg = small_cfg(dtype, B=3, pos_planes=3, n_sys=4, n_txt=6)
+    rng = np.random.default_rng(11)
+    n_vis, keeps = cfg.n_vis, (31, 16, 5)
+    S = cfg.n_sys + n_vis + cfg.n_txt
+    hidden = round_to_dtype(rng.standard_normal((cfg.B, S, cfg.Dh)).astype(np.float32), dtype)
+    pos = np.broadcast_to(np.arange(S, dtype=np.int32), (3, cfg.B, S)).copy()
+    pos[1] *= 2
+    h_ref, p_ref = hidden, pos
+    h_gpu, p_gpu = dev(hidden, dtype), dev(pos)
+    scale = float(cfg.d ** -0.5)
+    for layer, k_keep in enumerate(keeps):
+        S = cfg.n_sys + n_vis + cfg.n_txt
+        q = round_to_dtype(rng.standard_normal((cfg.B, cfg.Hq, cfg.d)).astype(np.float32), dtype)
+        k = round_to_dtype(rng.standard_normal((cfg.B, cfg.Hkv, S, cfg.d)).astype(np.float32), dtype)
+        v = round_to_dtype(rng.standard_normal((cfg.B, cfg.Hkv, S, cfg.d)).astype(np.float32), dtype)
+        plant.plant_stage2(cfg, q, k, scale, vo.SPAN_ONLY, n_vis=n_vis, k_keep=k_keep)
+        ref = [vo.llm_prune(q[b], k[b], v[b], h_ref[b], p_ref[:, b], cfg.n_sys, n_vis, cfg.n_txt, k_keep, scale)
+               for b in range(cfg.B)]
+        out = vs.vscan_llm_prune(dev(q, dtype), dev(k, dtype), dev(v, dtype), h_gpu, p_gpu, cfg.n_sys, n_vis,
+                                 cfg.n_txt, k_keep, scale)
+        h_ref = np.stack([r["hidden"] for r in ref])
+        p_ref = np.stack([r["pos"] for r in ref], axis=1)
+        np.testing.assert_array_equal(out["kept_vis"].cpu().numpy(), np.stack([r["kept_vis"] for r in ref]))
+        np.testing.assert_array_equal(out["hidden"].float().cpu().numpy(), h_ref)
+        np.testing.assert_array_equal(out["k"].float().cpu().numpy(), np.stack([r["k"] for r in ref]))
+        np.testing.assert_array_equal(out["v"].float().cpu().numpy(), np.stack([r["v"] for r in ref]))
+        np.testing.assert_array_equal(out["pos"].cpu().numpy(), p_ref)
+        h_gpu, p_gpu, n_vis = out["hidden"], out["pos"], k_keep
+    # plane 0 still holds original sequence positions: strictly increasing, system and text spans intact
+    final = p_gpu[0].cpu().numpy()
+    assert final.shape == (cfg.B, cfg.n_sys + keeps[-1] + cfg.n_txt) and np.all(np.diff(final, axis=1) > 0)
+    assert np.array_equal(final[:, :cfg.n_sys], np.tile(np.arange(cfg.n_sys), (cfg.B, 1)))
+    np.testing.assert_array_equal(p_gpu[1].cpu().numpy(), 2 * final)
 
 
 @pytest.mark.parametrize("k_keep,n_sys,n_txt", [(0, 3, 4), (20, 3, 4), (7, 0, 0), (20, 0, 5), (1, 2, 0)])

@@ -80,3 +80,23 @@ def test_planted_margins_hold():
 def test_tiny_config_is_consistent():
     t = tiny_config()
     assert t.N == 24 and t.W == 4 and t.K1 == 7 and t.n_vis == 14
+
+
+def test_schedule_points_follow_the_printed_settings():
+    """Table 1's (k, R2) pairs average 75 % of the Stage-1 set over 32 layers (App. B.1's rule), the
+    Table 6(a) pairs all average 11.1 %, and every schedule point is a legal call."""
+    from oracle import budget
+    from synth import schedule_points
+    from synth.configs import TABLE1_SETTINGS
+    for k, r2 in TABLE1_SETTINGS:
+        assert abs(budget.average_retention(1.0, r2 / 100, k, 32) - 0.75) < 1e-3
+    pts = schedule_points()
+    assert len(pts) == 12 + 5 + 5 + 1
+    for label, cfg, s1 in pts:
+        assert 0 <= cfg.k2 <= cfg.n_vis and cfg.k_w <= cfg.win_h * cfg.win_w and 0 <= cfg.k_g <= cfg.N - cfg.W * cfg.k_w
+        if label.startswith("table6a"):
+            assert abs(budget.average_tokens(cfg.K1, cfg.k2 // cfg.C, 16, 32) / cfg.N - 0.111) < 2e-3
+        if label.startswith("table6b"):
+            assert cfg.K1 == 96
+        if not s1:
+            assert cfg.n_vis == cfg.C * cfg.N
