@@ -14,14 +14,20 @@ import bench  # noqa: E402
 from synth import CONFIGS  # noqa: E402
 
 
-def test_algorithmic_bytes_match_the_scope_table():
-    # per image: 22.1 MB at the 2880-token shape, 12.8 MB at the 576-token batch shape, of which the
-    # compaction is 12.73 MB and 9.59 MB
+def test_algorithmic_bytes_count_every_byte_once():
+    # Per image at the 2880-token shape: attention rows 0.18 MB + head means and kept list 0.02 MB, features
+    # once and merged rows out 6.55 MB, keys of the visual span 2.63 MB, and the compaction's 12.73 MB of rows
+    # read and written less the 1.31 MB of surviving key rows that the scoring has already read: 20.8 MB.
     a2, a1 = bench.algorithmic_bytes(CONFIGS[2]), bench.algorithmic_bytes(CONFIGS[1])
-    assert abs(a2["step"] / 32 / 1e6 - 22.1) < 0.15
-    assert abs(a2["compact"] / 32 / 1e6 - 12.73) < 0.02
-    assert abs(a1["step"] / 256 / 1e6 - 12.8) < 0.15
-    assert abs(a1["compact"] / 256 / 1e6 - 9.59) < 0.02
+    assert abs(a2["step"] / 32 / 1e6 - 20.82) < 0.05
+    assert abs(a2["compact"] / 32 / 1e6 - (12.73 - 1.31)) < 0.02
+    assert abs(a2["qk_softmax"] / 32 / 1e6 - 2.63) < 0.01
+    assert a2["step"] == a2["score_select"] + a2["merge"] + a2["prune_fused"]
+    e, c = 2, CONFIGS[2]
+    survivors = c.B * c.Hkv * c.k2 * c.d * e
+    rows_moved = c.B * 2 * c.S_out * (c.Dh * e + 2 * c.Hkv * c.d * e + 4)
+    assert a2["compact"] == rows_moved - survivors
+    assert abs(a1["compact"] / 256 / 1e6 - (9.59 - 0.79)) < 0.02
     assert abs(bench.merge_flops(CONFIGS[2]) / 160 / 1e6 - 67.1) < 0.1
     assert abs(bench.merge_flops(CONFIGS[3]) / 4 / 1e9 - 75.2) < 0.1
 
