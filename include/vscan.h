@@ -59,10 +59,8 @@ typedef enum {
   VSCAN_MERGE_AUTO = 0,   /* bf16: INTERLEAVED for kept sets of 129..256, else TENSOR when the shape allows, else SIMT;
                              f32: SIMT */
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
-  VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group means in a
-                             second kernel */
-  VSCAN_MERGE_FUSED = 3,  /* norms, tcgen05 similarity + arg-max and group means in one kernel, one cluster of
-                             CTAs per instance (bf16, n_kept <= 256, n_tokens <= 8192) */
+  VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group sums in a second
+                             kernel, on the tensor cores too (one-hot matrix products) where the shape allows */
   VSCAN_MERGE_INTERLEAVED = 4 /* the TENSOR path's two steps in one persistent launch, one CTA per SM: six warps
                              assign tile after tile (kept rows packed and their norms taken by a small
                              kernel first), eight more warps sum the groups of every instance whose tiles are
@@ -186,7 +184,9 @@ vscan_status vscan_score_select(const vscan_score_select_desc* desc, void* strea
  * For every token u not in kept_idx: a(u) = argmax_s cos(m_u, m_kept[s]) (lowest slot on ties; norms
  * clamped at 1e-12), where m is `metric` if given, else x.  Then
  *   merged[b][s] = (x_kept[s] + sum_{a(u)=s} x_u) / (1 + |{u : a(u)=s}|),
- * accumulated in float32 in ascending token order and rounded once to `dtype`.
+ * accumulated in float32 and rounded once to `dtype` (CUDA-core sums add in ascending token order; sums on
+ * the tensor cores add tile by tile in the order of the hardware: the same result from run to run, not the
+ * same last bit as the CUDA-core path).
  *   x         [instances][row_len][dim] of `dtype`; row cls_offset + t is token t; rows before
  *             cls_offset (the [CLS] feature) are never read.  row_len >= cls_offset + n_tokens.
  *   metric    optional [instances][row_len][metric_dim] of `dtype`

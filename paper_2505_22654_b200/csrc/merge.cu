@@ -155,7 +155,8 @@ __global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergePara
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
   grid_dependency_wait();   // the assignments come from the kernel before this one
-  group_mean_body<T, VPL, R, kSlotsPerCta>(p, blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums);
+  group_mean_body<T, VPL, R, kSlotsPerCta, kSlotsPerCta>(p, blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums,
+                                                         static_cast<int>(threadIdx.x), CtaSync());
 }
 
 template <typename T, int VPL, int R>
@@ -206,7 +207,7 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
   if (!d || !d->x || !d->kept_idx || !d->merged) return VSCAN_ERR_INVALID_ARG;
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
   if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR &&
-      d->path != VSCAN_MERGE_FUSED && d->path != VSCAN_MERGE_INTERLEAVED)
+      d->path != VSCAN_MERGE_INTERLEAVED)
     return VSCAN_ERR_INVALID_ARG;
   if (d->instances < 0 || d->n_tokens <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + d->n_tokens ||
       d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
@@ -284,19 +285,6 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
   p.clear_status = 1;
 
-  // fused kernel: one launch for the whole call
-  if (d->path == VSCAN_MERGE_FUSED) {   // measured slower than the two-kernel tensor path: opt-in only
-    if (merge_fused_supported(d->dtype, p)) {
-      p.assign = d->assign;   // optional output only; the fused kernel keeps assignments on chip
-      VSCAN_CUDA_TRY(cudaMemsetAsync(p.status, 0, sizeof(uint32_t), stream));
-      st = launch_merge_fused(p, stream);
-      if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_FUSED) return st;
-      p.assign = d->assign ? d->assign : ws_assign;
-    } else if (d->path == VSCAN_MERGE_FUSED) {
-      return VSCAN_ERR_UNSUPPORTED;
-    }
-  }
-
   // assignment and group means in one persistent launch: on request, or by itself where it measured faster
   // than the two kernels below (kept sets above 128, where those run one or two CTAs per SM)
   if (d->path == VSCAN_MERGE_INTERLEAVED || (d->path == VSCAN_MERGE_AUTO && d->n_kept > 128)) {
@@ -332,6 +320,8 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   }
   // (Cutting the batch into runs of instances small enough for L2, so that the group-mean pass of a
   // run finds its features there, was measured slower: the smaller grids are latency-bound.)
-  return d->dtype == VSCAN_F32 ? launch_group_mean<float>(p, stream)
-                               : launch_group_mean<__nv_bfloat16>(p, stream);
+  if (d->dtype == VSCAN_F32) return launch_group_mean<float>(p, stream);
+  // after a tensor-core assignment the sums run on the tensor cores too where the shape allows
+  if (tensor && group_sum_tensor_supported(d->dtype, p)) return launch_group_sum_tensor(p, stream);
+  return launch_group_mean<__nv_bfloat16>(p, stream);
 }

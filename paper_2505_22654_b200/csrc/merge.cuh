@@ -32,9 +32,9 @@ bool assign_tensor_supported(int dtype, const MergeParams& p);
 // features from L2.  Clears the status word and uses the inv_norm region of the workspace for counters.
 vscan_status launch_merge_interleaved(const MergeParams& p, cudaStream_t stream);
 bool merge_interleaved_supported(int dtype, const MergeParams& p);
-// Norms, assignment and group means in one kernel (bf16, at most 256 kept tokens and 8192 tokens per
-// instance).  Writes merged / assign / counts directly; needs no inv_norm or assign scratch.
-vscan_status launch_merge_fused(const MergeParams& p, cudaStream_t stream);
-bool merge_fused_supported(int dtype, const MergeParams& p);
+// Group sums of Eq. 4 as one-hot matrix products on the tensor cores (bf16, at most 256 kept tokens, feature dim a
+// multiple of 128, no unused rows after the last token).  Reads `assign`, writes merged / counts.
+vscan_status launch_group_sum_tensor(const MergeParams& p, cudaStream_t stream);
+bool group_sum_tensor_supported(int dtype, const MergeParams& p);
 
 }  // namespace vscan

@@ -1,120 +1,157 @@
-// Group means of the merge step (Eq. 4): the body shared by the stand-alone group_mean kernel and by
-// the mean CTAs of the interleaved merge kernel.
+// Group means of the merge step (Eq. 4) on CUDA cores: the one body of the ordered sums, shared by the stand-alone
+// group_mean kernel and by the mean warps of the persistent merge kernel, and the bit-mask variant for short instances.
 #pragma once
 
 #include "merge.cuh"
 
 namespace vscan {
 
-// One CTA per (group of slots, instance), one warp per slot: 4 slots per CTA for short instances, 16
-// for long ones (the list-building prologue is O(n_tokens) per CTA); warp w owns slot s0 + w.  The CTA first lists, in
-// ascending token order, the tokens assigned to its slots; each warp then walks that list and adds
-// its members' rows in that order (fp32), R rows in flight.  Small CTAs keep a large group from
-// holding the resources of many finished warps.
-// dynamic shared memory: list[n_tokens] of (local slot << 24 | token), then assign[n_tokens]
-// `list` is shared memory of 2 * n_tokens words: list[n_tokens] of (local slot << 24 | token), then assign[n_tokens];
-// `warp_sums` is shared scratch of 33 ints.  Called by all kSlotsPerCta * 32 threads of the CTA.
-template <typename T, int VPL, int R, int kSlotsPerCta>
-__device__ __forceinline__ void group_mean_body(const MergeParams& p, int b, int s0, uint32_t* list, int* warp_sums) {
-  constexpr int kMeanThreads = kSlotsPerCta * 32;
+// How the threads that share a group-mean job meet: the whole CTA, or a subset of its warps on a named barrier.
+struct CtaSync {
+  __device__ __forceinline__ void operator()() const { __syncthreads(); }
+};
+template <int kBarrier, int kThreadsOfGroup>
+struct NamedSync {
+  __device__ __forceinline__ void operator()() const { asm volatile("bar.sync %0, %1;" ::"n"(kBarrier), "n"(kThreadsOfGroup) : "memory"); }
+};
+
+// Exclusive prefix sum of one int per thread over the kWarps warps of a group; `total` gets the group sum.
+// `warp_sums` is shared scratch of at least 33 ints.
+template <int kWarps, typename Sync>
+__device__ __forceinline__ int group_exclusive_scan(int v, int* warp_sums, int& total, int gwarp, int lane, Sync sync) {
+  int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  sync();   // protect warp_sums from a previous use
+  if (lane == 31) warp_sums[gwarp] = incl;
+  sync();
+  if (gwarp == 0) {
+    const int w = lane < kWarps ? warp_sums[lane] : 0;
+    int wi = w;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
+    }
+    if (lane < kWarps) warp_sums[lane] = wi - w;
+    if (lane == 31) warp_sums[32] = wi;
+  }
+  sync();
+  total = warp_sums[32];
+  return warp_sums[gwarp] + incl - v;
+}
+
+// The ordered group sums of Eq. 4 for kSlots consecutive kept slots s0 .. s0 + kSlots - 1 of instance b, by a group
+// of kWarps warps (thread `gtid` of the group): the stand-alone group_mean kernel calls it with its whole CTA, the
+// persistent merge kernel with its mean warps.  The group first lists, in ascending token order, the tokens
+// assigned to its slots; warp w then takes slots w, w + kWarps, ..., walks the list and adds the members' rows in
+// that order (fp32), R rows in flight, VPL 16-byte pieces per lane and column pass; one rounding on output.
+// `list` is shared memory of 2 * n_tokens words: list[n_tokens] of (local slot << 24 | token), then
+// assign[n_tokens]; `warp_sums` is shared scratch of 33 ints.
+template <typename T, int VPL, int R, int kSlots, int kWarps, typename Sync>
+__device__ __forceinline__ void group_mean_body(const MergeParams& p, int b, int s0, uint32_t* list, int* warp_sums,
+                                                int gtid, Sync sync) {
+  constexpr int kGroupThreads = kWarps * 32;
   constexpr int E = Vec16<T>::kElems;
-  // all assignments of the instance -> shared memory (second half of the buffer) in one round of
+  const int gwarp = gtid >> 5, lane = gtid & 31;
+  // all assignments of the instance -> shared memory (second half of the buffer) in rounds of
   // independent, coalesced loads; the two ordered passes below then run out of shared memory
   int32_t* assign = reinterpret_cast<int32_t*>(list + p.n_tokens);
   {
     const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
-    for (int i0 = threadIdx.x; i0 < p.n_tokens; i0 += kMeanThreads * 8) {
+    for (int i0 = gtid; i0 < p.n_tokens; i0 += kGroupThreads * 8) {
       int32_t v[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
+      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kGroupThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kMeanThreads; if (i < p.n_tokens) assign[i] = v[u]; }
+      for (int u = 0; u < 8; ++u) { const int i = i0 + u * kGroupThreads; if (i < p.n_tokens) assign[i] = v[u]; }
     }
   }
-  __syncthreads();
+  sync();
 
   // contiguous run of tokens per thread; an odd run length keeps the threads of a warp on different banks
-  const int per = ((p.n_tokens + blockDim.x - 1) / blockDim.x) | 1;
-  const int lo = min(p.n_tokens, static_cast<int>(threadIdx.x) * per), hi = min(p.n_tokens, lo + per);
+  const int per = ((p.n_tokens + kGroupThreads - 1) / kGroupThreads) | 1;
+  const int lo = min(p.n_tokens, gtid * per), hi = min(p.n_tokens, lo + per);
   int mine = 0;
-  for (int i = lo; i < hi; ++i) {
-    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
-    mine += rel < static_cast<unsigned>(kSlotsPerCta);
-  }
+  for (int i = lo; i < hi; ++i) mine += static_cast<unsigned>(assign[i] - s0) < static_cast<unsigned>(kSlots);
   int n_list;
-  int pos = block_exclusive_scan(mine, warp_sums, n_list);
+  int pos = group_exclusive_scan<kWarps>(mine, warp_sums, n_list, gwarp, lane, sync);
   for (int i = lo; i < hi; ++i) {
     const unsigned rel = static_cast<unsigned>(assign[i] - s0);
-    if (rel < static_cast<unsigned>(kSlotsPerCta)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
+    if (rel < static_cast<unsigned>(kSlots)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
   }
-  __syncthreads();
+  sync();
 
-  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31, s = s0 + w;
-  if (s >= p.n_kept) return;
   const int vecs = p.dim / E;
   const T* xb = static_cast<const T*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
-  T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
-
-  for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
-    float acc[VPL][E];
+  for (int sl = gwarp; sl < kSlots; sl += kWarps) {
+    const int s = s0 + sl;
+    if (s >= p.n_kept) break;
+    T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
+    for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
+      float acc[VPL][E];
 #pragma unroll
-    for (int i = 0; i < VPL; ++i)
+      for (int i = 0; i < VPL; ++i)
 #pragma unroll
-      for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
-    int count = 0;
-    for (int c = 0; c < n_list; c += 32) {
-      const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
-      unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(w));
-      count += __popc(mask);
-      while (mask) {
-        int tok[R];
+        for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+      int count = 0;
+      for (int c = 0; c < n_list; c += 32) {
+        const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
+        unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(sl));
+        count += __popc(mask);
+        while (mask) {
+          int tok[R];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          tok[r] = -1;
-          if (mask) {
-            const int l = __ffs(mask) - 1;
-            mask &= mask - 1;
-            tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
+          for (int r = 0; r < R; ++r) {
+            tok[r] = -1;
+            if (mask) {
+              const int l = __ffs(mask) - 1;
+              mask &= mask - 1;
+              tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
+            }
           }
-        }
-        uint4 raw[R][VPL];
+          uint4 raw[R][VPL];
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
+          for (int r = 0; r < R; ++r) {
+            const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
 #pragma unroll
-          for (int i = 0; i < VPL; ++i) {
-            const int v = v0 + lane + 32 * i;
-            if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
+            for (int i = 0; i < VPL; ++i) {
+              const int v = v0 + lane + 32 * i;
+              if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
+            }
           }
-        }
 #pragma unroll
-        for (int r = 0; r < R; ++r) {
-          if (tok[r] < 0) continue;
+          for (int r = 0; r < R; ++r) {
+            if (tok[r] < 0) continue;
 #pragma unroll
-          for (int i = 0; i < VPL; ++i) {
-            const int v = v0 + lane + 32 * i;
-            if (v < vecs) {
-              float f[E];
-              Vec16<T>::unpack(raw[r][i], f);
+            for (int i = 0; i < VPL; ++i) {
+              const int v = v0 + lane + 32 * i;
+              if (v < vecs) {
+                float f[E];
+                Vec16<T>::unpack(raw[r][i], f);
 #pragma unroll
-              for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+                for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+              }
             }
           }
         }
       }
-    }
-    const float inv = 1.f / static_cast<float>(max(count, 1));
+      const float inv = 1.f / static_cast<float>(max(count, 1));
 #pragma unroll
-    for (int i = 0; i < VPL; ++i) {
-      const int v = v0 + lane + 32 * i;
-      if (v < vecs) {
-        float f[E];
+      for (int i = 0; i < VPL; ++i) {
+        const int v = v0 + lane + 32 * i;
+        if (v < vecs) {
+          float f[E];
 #pragma unroll
-        for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
-        st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
+          for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
+          st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
+        }
       }
+      if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
     }
-    if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
   }
 }
 

@@ -14,6 +14,7 @@
 #include <cstdlib>
 
 #include "merge.cuh"
+#include "merge_mean.cuh"
 #include "tc_common.cuh"
 
 namespace vscan {
@@ -314,133 +315,6 @@ struct PersistShared {
 
 __device__ __forceinline__ void mean_group_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kMeanThreads) : "memory"); }
 
-// Exclusive prefix sum over the 256 threads of the mean group (named barrier 2).
-__device__ __forceinline__ int mean_group_scan(int v, int* warp_sums, int& total, int gwarp, int lane) {
-  int incl = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  mean_group_sync();   // protect warp_sums from a previous use
-  if (lane == 31) warp_sums[gwarp] = incl;
-  mean_group_sync();
-  if (gwarp == 0) {
-    const int w = lane < kMeanWarps ? warp_sums[lane] : 0;
-    int wi = w;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, wi, o);
-      if (lane >= o) wi += t;
-    }
-    if (lane < kMeanWarps) warp_sums[lane] = wi - w;
-    if (lane == 31) warp_sums[32] = wi;
-  }
-  mean_group_sync();
-  total = warp_sums[32];
-  return warp_sums[gwarp] + incl - v;
-}
-
-// One mean job: slots s0 .. s0 + kJobSlots - 1 of instance b.  `list`: 2 * n_tokens words of shared memory.
-template <int VPL, int R>
-__device__ __forceinline__ void mean_job(const MergeParams& p, int b, int s0, uint32_t* list, int* warp_sums, int gtid) {
-  constexpr int E = 8;
-  const int gwarp = gtid >> 5, lane = gtid & 31;
-  int32_t* assign = reinterpret_cast<int32_t*>(list + p.n_tokens);
-  {
-    const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
-    for (int i0 = gtid; i0 < p.n_tokens; i0 += kMeanThreads * 4) {
-      int32_t v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) { const int i = i0 + u * kMeanThreads; v[u] = i < p.n_tokens ? __ldcg(ag + i) : 0; }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) { const int i = i0 + u * kMeanThreads; if (i < p.n_tokens) assign[i] = v[u]; }
-    }
-  }
-  mean_group_sync();
-  // contiguous run of tokens per thread; an odd run length keeps the threads of a warp on different banks
-  const int per = ((p.n_tokens + kMeanThreads - 1) / kMeanThreads) | 1;
-  const int lo = min(p.n_tokens, gtid * per), hi = min(p.n_tokens, lo + per);
-  int mine = 0;
-  for (int i = lo; i < hi; ++i) mine += static_cast<unsigned>(assign[i] - s0) < static_cast<unsigned>(kJobSlots);
-  int n_list;
-  int pos = mean_group_scan(mine, warp_sums, n_list, gwarp, lane);
-  for (int i = lo; i < hi; ++i) {
-    const unsigned rel = static_cast<unsigned>(assign[i] - s0);
-    if (rel < static_cast<unsigned>(kJobSlots)) list[pos++] = (rel << 24) | static_cast<unsigned>(i);
-  }
-  mean_group_sync();
-
-  const int vecs = p.dim / E;
-  const __nv_bfloat16* xb = static_cast<const __nv_bfloat16*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
-  for (int sl = gwarp; sl < kJobSlots; sl += kMeanWarps) {
-    const int s = s0 + sl;
-    if (s >= p.n_kept) break;
-    __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
-    for (int v0 = 0; v0 < vecs; v0 += 32 * VPL) {
-      float acc[VPL][E];
-#pragma unroll
-      for (int i = 0; i < VPL; ++i)
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
-      int count = 0;
-      for (int c = 0; c < n_list; c += 32) {
-        const uint32_t entry = c + lane < n_list ? list[c + lane] : 0xFFFFFFFFu;
-        unsigned mask = __ballot_sync(0xffffffffu, (entry >> 24) == static_cast<unsigned>(sl));
-        count += __popc(mask);
-        while (mask) {
-          int tok[R];
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            tok[r] = -1;
-            if (mask) {
-              const int l = __ffs(mask) - 1;
-              mask &= mask - 1;
-              tok[r] = static_cast<int>(__shfl_sync(0xffffffffu, entry, l) & 0xFFFFFFu);
-            }
-          }
-          uint4 raw[R][VPL];
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok[r] < 0 ? tok[0] : tok[r]) * p.dim);
-#pragma unroll
-            for (int i = 0; i < VPL; ++i) {
-              const int v = v0 + lane + 32 * i;
-              if (v < vecs && tok[r] >= 0) raw[r][i] = ld_nc_16(row + v);
-            }
-          }
-#pragma unroll
-          for (int r = 0; r < R; ++r) {
-            if (tok[r] < 0) continue;
-#pragma unroll
-            for (int i = 0; i < VPL; ++i) {
-              const int v = v0 + lane + 32 * i;
-              if (v < vecs) {
-                float f[E];
-                Vec16<__nv_bfloat16>::unpack(raw[r][i], f);
-#pragma unroll
-                for (int e = 0; e < E; ++e) acc[i][e] += f[e];
-              }
-            }
-          }
-        }
-      }
-      const float inv = 1.f / static_cast<float>(max(count, 1));
-#pragma unroll
-      for (int i = 0; i < VPL; ++i) {
-        const int v = v0 + lane + 32 * i;
-        if (v < vecs) {
-          float f[E];
-#pragma unroll
-          for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
-          st_16(reinterpret_cast<uint4*>(out) + v, Vec16<__nv_bfloat16>::pack(f));
-        }
-      }
-      if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
-    }
-  }
-}
-
 // Packs the kept rows like pack_kept_kernel and, having read them anyway, writes 1 / max(|m_s|, eps) of every
 // kept token; the first CTA also zeroes the status word and the counters of the persistent kernel that
 // follows.  One warp per slot, the whole row in flight at once.
@@ -675,7 +549,9 @@ merge_persistent_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_
       const int q = shp.job, ready = shp.ready;
       mean_group_sync();   // everyone has the job before thread 0 takes the next one
       if (q >= ps.total_jobs || !ready) break;
-      mean_job<4, 4>(m, q / ps.jobs_per_instance, (q % ps.jobs_per_instance) * kJobSlots, mean_list, shp.warp_sums, gtid);
+      // the ordered sums of group_mean_kernel: same additions in the same order, hence the same bits
+      group_mean_body<__nv_bfloat16, 4, 4, kJobSlots, kMeanWarps>(m, q / ps.jobs_per_instance, (q % ps.jobs_per_instance) * kJobSlots,
+                                                                  mean_list, shp.warp_sums, gtid, NamedSync<2, kMeanThreads>());
     }
   }
 

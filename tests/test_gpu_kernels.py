@@ -166,7 +166,7 @@ def test_merge_exact_ties_and_duplicates():
 
 @pytest.mark.parametrize("N,D,K1,c", [(576, 1024, 64, 1), (576, 1024, 192, 1), (300, 72, 17, 0), (130, 264, 130, 1),
                                       (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0)])
-@pytest.mark.parametrize("path", ["tensor", "fused", "interleaved"])
+@pytest.mark.parametrize("path", ["tensor", "interleaved"])
 def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     """The tcgen05 path on its own (path = TENSOR): tile tails, kept counts that are not multiples of
     16, more than 256 kept tokens (several accumulator rounds), feature dims that are not multiples
@@ -175,11 +175,6 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     x = round_to_dtype(RNG.standard_normal((2, N + c, D)).astype(np.float32), "bf16")
     kept = np.stack([np.sort(RNG.choice(N, K1, replace=False)) for _ in range(2)])
     plant.plant_merge(cfg, x, kept)
-    if path == "fused" and K1 > 256:
-        with pytest.raises(vs.VScanError) as e:
-            vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_FUSED)
-        assert e.value.status == 2       # more kept tokens than one accumulator holds: not this path
-        return
     if path == "interleaved" and K1 > 256:
         with pytest.raises(vs.VScanError) as e:
             vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), path=vs.MERGE_INTERLEAVED)
@@ -188,8 +183,7 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     ws = vs.Workspace(8 << 20)
     merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
                                             want_counts=True, workspace=ws,
-                                            path={"tensor": vs.MERGE_TENSOR, "fused": vs.MERGE_FUSED,
-                                                  "interleaved": vs.MERGE_INTERLEAVED}[path])
+                                            path={"tensor": vs.MERGE_TENSOR, "interleaved": vs.MERGE_INTERLEAVED}[path])
     assert vs.vscan_check(ws) == 0
     for b in range(2):
         m, a, cn = vo.merge(x[b], c, kept[b])
@@ -216,8 +210,11 @@ def test_merge_interleaved_many_instances(B, N, D, K1):
         same = (ref[1] == out[1]).all(dim=1)      # (the two paths round the kept-row norms in different orders:
         assert same.float().mean() > 0.9          #  a near-tie may fall the other way)
         assert (ref[1] == out[1]).float().mean() > 0.999
-        for r, o in zip(ref, out):
-            assert torch.equal(r[same], o[same])
+        assert torch.equal(ref[1][same], out[1][same]) and torch.equal(ref[2][same], out[2][same])
+        # the two paths add a group's rows in different orders (tensor-core sums against ordered fp32 sums):
+        # the same means up to the last bf16 digit
+        a, c = ref[0][same].float(), out[0][same].float()
+        assert bool(((a - c).abs() <= 2.0 ** -7 * torch.maximum(a.abs(), c.abs()) + 1e-6).all())
     for b in (0, B // 2, B - 1):                  # unplanted inputs: the near-tie rule decides what may differ
         n_band = check_merge_unplanted(x[b], 0, kept[b], out[0][b], out[1][b], out[2][b], "bf16")
         assert n_band <= N // 20

@@ -49,7 +49,7 @@ def test_random_stage1(seed):
     # merge on those kept tokens, every path the dtype allows
     x = round_to_dtype(rng.standard_normal((B, N + c, D)).astype(np.float32), dtype)
     plant.plant_merge(cfg, x, ref)
-    paths = [vs.MERGE_AUTO, vs.MERGE_SIMT] + ([vs.MERGE_TENSOR, vs.MERGE_FUSED] if dtype == "bf16" and ref.shape[1] <= 256 else [])
+    paths = [vs.MERGE_AUTO, vs.MERGE_SIMT] + ([vs.MERGE_TENSOR, vs.MERGE_INTERLEAVED] if dtype == "bf16" and ref.shape[1] <= 256 else [])
     if dtype == "bf16" and ref.shape[1] <= 128:
         paths.append(vs.MERGE_INTERLEAVED)
     for path in paths:
