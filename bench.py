@@ -437,6 +437,9 @@ def run_sweep(args, rank, world, local_rank, dist):
     points += [(label, cfg, 0, s1) for label, cfg, s1 in schedule_points()]
     if args.sweep_filter:
         points = [p for p in points if args.sweep_filter in p[0]]
+    if rank == 0 and (not args.sweep_filter or args.sweep_filter in "ragged"):
+        import torch
+        print(json.dumps(measure_ragged(args, torch.device("cuda", local_rank))), flush=True)
     for label, cfg, path, s1 in points:
         args.merge_path = path
         steps = args.steps
@@ -456,6 +459,52 @@ def run_sweep(args, rank, world, local_rank, dist):
                "kernels_us": {n: round(v["avg_us"] * v["launches_per_step"], 1) for n, v in k.items()},
                "clocks_mhz": line["clocks"]["sm_mhz"], "reasons": line["clocks"]["reasons"]}
         print(json.dumps(out), flush=True)
+
+
+def measure_ragged(args, device):
+    """One mixed-resolution batch through the ragged entry points (dynamic-resolution shapes, Sec. 5.1 "Models"):
+    instances of 576 to 16384 tokens sorted by size, 11.1 % of each kept, then sequences of matching lengths pruned
+    to half.  CUDA events over repeated calls; inputs (63 MB + 1.1 GB) rotate through three packed copies."""
+    import torch
+
+    from paper_2505_22654_b200 import binding as vb
+    dt, D, H, Hq, Hkv, d, Dh = torch.bfloat16, 1280, 16, 28, 4, 128, 3584
+    mix = [(1, 24, 24)] * 8 + [(1, 32, 32)] * 8 + [(1, 48, 48)] * 4 + [(4, 32, 32)] * 2 + [(9, 32, 32)] + [(16, 32, 32)]
+    g = torch.Generator(device="cpu").manual_seed(0)
+    toks = [f * a * b for f, a, b in mix]
+    kw = [1] * len(mix)                                                   # one local token per 4 x 4 window
+    kg = [max(1, round(0.111 * n) - n // 16) for n in toks]               # the rest of the 11.1 % globally
+    k1 = [n // 16 + k for n, k in zip(toks, kg)]
+    attn = [torch.softmax(3 * torch.randn((H, n), generator=g), dim=-1).to(dt).to(device) for n in toks]
+    xs = [torch.randn((n, D), generator=g).to(dt).to(device) for n in toks]
+    n_sys, n_txt = [0] * len(mix), [128] * len(mix)
+    k2 = [k // 2 for k in k1]
+    q = torch.randn((len(mix), Hq, d), generator=g).to(dt).to(device)
+    ks = [(torch.randn((Hkv, k + 128, d), generator=g) * d ** -0.5).to(dt).to(device) for k in k1]
+    hs = [torch.randn((k + 128, Dh), generator=g).to(dt).to(device) for k in k1]
+    ps = [torch.arange(k + 128, dtype=torch.int32, device=device) for k in k1]
+    stream = torch.cuda.Stream(device)
+    with torch.cuda.stream(stream):
+        def step():
+            _, _, w1 = vb.vscan_stage1_ragged(attn, attn, xs, 0, mix, 4, 4, kw, kg)
+            _, w2 = vb.vscan_llm_prune_ragged(q, ks, ks, hs, ps, n_sys, k1, n_txt, k2, d ** -0.5)
+            return w1, w2
+        before = vb.kernel_launches()
+        w1, w2 = step()
+        launches = vb.kernel_launches() - before
+        stream.synchronize()
+        n = 10
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            w1, w2 = step()
+        e1.record(stream)
+        e1.synchronize()
+        status = max(vb.vscan_check(w1), vb.vscan_check(w2))
+    ms = e0.elapsed_time(e1) / n
+    return {"point": "ragged: 24 images of 576..16384 tokens in one call per stage (packing by the binding included)",
+            "images": len(mix), "tokens": sum(toks), "kept": sum(k1), "ms_per_call_pair": round(ms, 3),
+            "images_per_s": round(len(mix) / (ms * 1e-3), 1), "kernel_launches": launches, "status": status}
 
 
 def main():

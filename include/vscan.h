@@ -25,8 +25,9 @@
  *     (VSCAN_F32 or VSCAN_BF16).  Scores are always float32, indices int32.
  *   - Ties: wherever a top-k or an arg-max meets equal values the lowest index wins.  Survivor
  *     lists are in ascending original index.
- *   - Shapes are uniform over the batch of one call.  Counts (k_global, k_per_window, k_keep) are
- *     explicit integers; percentages (R1, R2 of the paper) are resolved by the caller.
+ *   - Shapes are uniform over the batch of one call (mixed sizes: the *_ragged entry points).  Counts
+ *     (k_global, k_per_window, k_keep) are explicit integers; percentages (R1, R2 of the paper) are
+ *     resolved by the caller.
  */
 #ifndef VSCAN_H_
 #define VSCAN_H_
@@ -257,6 +258,91 @@ typedef struct {
 size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* desc);
 vscan_status vscan_llm_prune(const vscan_prune_desc* desc, void* workspace, size_t workspace_bytes,
                              void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Ragged batches (Sec. 5.1 "Models": encoders with dynamic resolution hand over between 4 and 16384 visual
+ * tokens per image; Sec. 4.1 and 4.2 are per instance and per sequence, so units of different sizes are
+ * independent problems).
+ *
+ * One call for instances (vscan_stage1_ragged: Eq. 2 + Eq. 3 selection, then the Eq. 4 merge) or sequences
+ * (vscan_llm_prune_ragged: Sec. 4.2) whose sizes differ.  Every result is the one the uniform entry points give
+ * for that unit alone.
+ *   - The size, budget and offset arrays are HOST arrays with one entry per unit (the caller derives them from
+ *     the image resolutions); they are read during the call and not kept.  Tensors are packed DEVICE buffers;
+ *     unit i's block starts at the given ELEMENT offset of its buffer and has the uniform layout of that
+ *     tensor for a batch of one.  Every block must start on a 16-byte boundary.
+ *   - The library cuts the batch into runs of consecutive units with equal shape, equal budgets and regularly
+ *     spaced blocks and enqueues the uniform kernels once per run on `stream`: a batch sorted by size costs
+ *     one set of launches per distinct size, a batch of all-different sizes one set per unit.
+ *   - Workspace: vscan_*_ragged_workspace_bytes(desc); vscan_check(workspace, stream) reports a bounded wait
+ *     that ran out in any run.  Everything is validated before the first launch.
+ * vscan_stage1_ragged
+ *   attn_global, attn_local  per instance [heads][cls_offset + N_i] at attn_offset[i] (the two may be one buffer)
+ *   x                        per instance [cls_offset + N_i][dim] at x_offset[i]
+ *   kept_idx (out)           per instance [K1_i] at kept_offset[i], K1_i = windows_i * k_per_window[i] + k_global[i] >= 1
+ *   merged (out)             per instance [K1_i][dim] at kept_offset[i] * dim
+ *   N_i = frames[i] * grid_h[i] * grid_w[i] <= 16384; win_h | grid_h[i], win_w | grid_w[i]
+ * vscan_llm_prune_ragged   (fields as in vscan_prune_desc, per sequence)
+ *   q_last [batch][q_heads][head_dim] (uniform);  k, v per sequence [kv_heads][S_i][head_dim] at kv_offset[i];
+ *   hidden [S_i][hidden_dim] at hidden_offset[i];  pos_ids [S_i] at pos_offset[i] (one plane);
+ *   kept_vis (out) [k_keep[i]] at kept_offset[i];  k_out, v_out [kv_heads][S'_i][head_dim] at kv_out_offset[i];
+ *   hidden_out [S'_i][hidden_dim] at hidden_out_offset[i];  pos_out [S'_i] at pos_out_offset[i];
+ *   S_i = n_sys[i] + n_vis[i] + n_txt[i], S'_i = S_i - n_vis[i] + k_keep[i].  v / hidden / pos_ids optional as pairs.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t dtype;      /* vscan_dtype */
+  int32_t merge_path; /* vscan_merge_path */
+  int32_t instances, heads, cls_offset, dim, win_h, win_w;
+  const void* attn_global;
+  const void* attn_local;
+  const void* x;
+  int32_t* kept_idx;
+  void* merged;
+  const int32_t* frames;       /* host arrays [instances] from here on */
+  const int32_t* grid_h;
+  const int32_t* grid_w;
+  const int32_t* k_per_window;
+  const int32_t* k_global;
+  const int64_t* attn_offset;
+  const int64_t* x_offset;
+  const int64_t* kept_offset;
+} vscan_stage1_ragged_desc;
+
+size_t vscan_stage1_ragged_workspace_bytes(const vscan_stage1_ragged_desc* desc);
+vscan_status vscan_stage1_ragged(const vscan_stage1_ragged_desc* desc, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+
+typedef struct {
+  int32_t dtype; /* vscan_dtype */
+  int32_t batch, q_heads, kv_heads, head_dim, hidden_dim, pos_planes;
+  int32_t softmax_span; /* vscan_softmax_span */
+  float scale;
+  const void* q_last;
+  const void* k;
+  const void* v;
+  const void* hidden;
+  const int32_t* pos_ids;
+  int32_t* kept_vis;
+  void* hidden_out;
+  void* k_out;
+  void* v_out;
+  int32_t* pos_out;
+  const int32_t* n_sys;        /* host arrays [batch] from here on */
+  const int32_t* n_vis;
+  const int32_t* n_txt;
+  const int32_t* k_keep;
+  const int64_t* kv_offset;
+  const int64_t* kv_out_offset;
+  const int64_t* hidden_offset;
+  const int64_t* hidden_out_offset;
+  const int64_t* pos_offset;
+  const int64_t* pos_out_offset;
+  const int64_t* kept_offset;
+} vscan_prune_ragged_desc;
+
+size_t vscan_llm_prune_ragged_workspace_bytes(const vscan_prune_ragged_desc* desc);
+vscan_status vscan_llm_prune_ragged(const vscan_prune_ragged_desc* desc, void* workspace, size_t workspace_bytes,
+                                    void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Housekeeping.

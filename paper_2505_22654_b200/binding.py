@@ -57,6 +57,26 @@ class PruneDesc(C.Structure):
                 ("pos_out", _vp), ("scores", _vp)]
 
 
+_i64p, _i32p = C.POINTER(C.c_int64), C.POINTER(C.c_int32)
+
+
+class Stage1RaggedDesc(C.Structure):
+    _fields_ = [("dtype", _i32), ("merge_path", _i32), ("instances", _i32), ("heads", _i32), ("cls_offset", _i32),
+                ("dim", _i32), ("win_h", _i32), ("win_w", _i32), ("attn_global", _vp), ("attn_local", _vp), ("x", _vp),
+                ("kept_idx", _vp), ("merged", _vp), ("frames", _i32p), ("grid_h", _i32p), ("grid_w", _i32p),
+                ("k_per_window", _i32p), ("k_global", _i32p), ("attn_offset", _i64p), ("x_offset", _i64p),
+                ("kept_offset", _i64p)]
+
+
+class PruneRaggedDesc(C.Structure):
+    _fields_ = [("dtype", _i32), ("batch", _i32), ("q_heads", _i32), ("kv_heads", _i32), ("head_dim", _i32),
+                ("hidden_dim", _i32), ("pos_planes", _i32), ("softmax_span", _i32), ("scale", _f32), ("q_last", _vp),
+                ("k", _vp), ("v", _vp), ("hidden", _vp), ("pos_ids", _vp), ("kept_vis", _vp), ("hidden_out", _vp),
+                ("k_out", _vp), ("v_out", _vp), ("pos_out", _vp), ("n_sys", _i32p), ("n_vis", _i32p), ("n_txt", _i32p),
+                ("k_keep", _i32p), ("kv_offset", _i64p), ("kv_out_offset", _i64p), ("hidden_offset", _i64p),
+                ("hidden_out_offset", _i64p), ("pos_offset", _i64p), ("pos_out_offset", _i64p), ("kept_offset", _i64p)]
+
+
 class VScanError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -87,6 +107,11 @@ def lib() -> C.CDLL:
         for fn, desc in (("vscan_score", ScoreDesc), ("vscan_select_global_local", SelectDesc),
                          ("vscan_merge", MergeDesc), ("vscan_llm_prune", PruneDesc)):
             f = getattr(L, fn)
+            f.restype, f.argtypes = _i32, [C.POINTER(desc), _vp, C.c_size_t, _vp]
+        for name, desc in (("stage1_ragged", Stage1RaggedDesc), ("llm_prune_ragged", PruneRaggedDesc)):
+            ws = getattr(L, f"vscan_{name}_workspace_bytes")
+            ws.restype, ws.argtypes = C.c_size_t, [C.POINTER(desc)]
+            f = getattr(L, f"vscan_{name}")
             f.restype, f.argtypes = _i32, [C.POINTER(desc), _vp, C.c_size_t, _vp]
         L.vscan_score_select.restype = _i32
         L.vscan_score_select.argtypes = [C.POINTER(ScoreSelectDesc), _vp]
@@ -309,6 +334,111 @@ def vscan_llm_prune(q_last, k, v, hidden, pos_ids, n_sys, n_vis, n_txt, k_keep, 
                      v_out=_ptr(o.get("v")), pos_out=_ptr(o.get("pos")), scores=_ptr(o.get("scores")))
     _call("vscan_llm_prune", desc, "vscan_llm_prune_workspace_bytes", workspace)
     return o
+
+
+# ------------------------------------------------------------------------------------------ ragged batches
+def _host_i32(values):
+    return (C.c_int32 * len(values))(*[int(v) for v in values])
+
+
+def _host_i64(values):
+    return (C.c_int64 * len(values))(*[int(v) for v in values])
+
+
+def _aligned_offsets(sizes, align_elems):
+    """Element offsets of consecutive blocks, each block starting on a multiple of `align_elems`."""
+    offs, cur = [], 0
+    for n in sizes:
+        cur = -(-cur // align_elems) * align_elems
+        offs.append(cur)
+        cur += int(n)
+    return offs, cur
+
+
+def vscan_stage1_ragged(attn_g_list, attn_l_list, x_list, cls_offset, grids, win_h, win_w, k_per_window, k_global,
+                        path=MERGE_AUTO, workspace=None):
+    """Stage 1 for instances of different sizes in one library call.  attn_*_list[i]: [H, c + N_i], x_list[i]:
+    [c + N_i, D] (CUDA tensors); grids[i] = (frames, grid_h, grid_w); k_per_window / k_global: per-instance lists.
+    Packs the inputs (argument marshalling only) and returns ([kept_idx_i], [merged_i]) as views of the packed
+    outputs, plus the workspace (for vscan_check)."""
+    n = len(x_list)
+    dt, dev = x_list[0].dtype, x_list[0].device
+    e_align = 16 // x_list[0].element_size()
+    H, D = attn_g_list[0].shape[0], x_list[0].shape[1]
+    a_off, a_total = _aligned_offsets([t.numel() for t in attn_g_list], e_align)
+    x_off, x_total = _aligned_offsets([t.numel() for t in x_list], e_align)
+    k1 = [f * (gh // win_h) * (gw // win_w) * kw + kg for (f, gh, gw), kw, kg in zip(grids, k_per_window, k_global)]
+    # kept lists are int32 (4 per 16 bytes); merged rows start at kept_offset * D, so 4-entry alignment covers both
+    k_off, k_total = _aligned_offsets(k1, 4 if (4 * D * x_list[0].element_size()) % 16 == 0 else 16)
+    ag = torch.zeros(a_total, dtype=dt, device=dev)
+    al = torch.zeros(a_total, dtype=dt, device=dev)
+    x = torch.zeros(x_total, dtype=dt, device=dev)
+    for i in range(n):
+        ag[a_off[i]:a_off[i] + attn_g_list[i].numel()] = attn_g_list[i].reshape(-1)
+        al[a_off[i]:a_off[i] + attn_l_list[i].numel()] = attn_l_list[i].reshape(-1)
+        x[x_off[i]:x_off[i] + x_list[i].numel()] = x_list[i].reshape(-1)
+    kept = torch.full((max(k_total, 1),), -1, dtype=torch.int32, device=dev)
+    merged = torch.zeros((max(k_total, 1) * D,), dtype=dt, device=dev)
+    keep_alive = [_host_i32([g[0] for g in grids]), _host_i32([g[1] for g in grids]), _host_i32([g[2] for g in grids]),
+                  _host_i32(k_per_window), _host_i32(k_global), _host_i64(a_off), _host_i64(x_off), _host_i64(k_off)]
+    d = Stage1RaggedDesc(dtype=_dtype_code(x), merge_path=path, instances=n, heads=H, cls_offset=cls_offset, dim=D,
+                         win_h=win_h, win_w=win_w, attn_global=_ptr(ag), attn_local=_ptr(al), x=_ptr(x),
+                         kept_idx=_ptr(kept), merged=_ptr(merged), frames=keep_alive[0], grid_h=keep_alive[1],
+                         grid_w=keep_alive[2], k_per_window=keep_alive[3], k_global=keep_alive[4],
+                         attn_offset=keep_alive[5], x_offset=keep_alive[6], kept_offset=keep_alive[7])
+    workspace = _call("vscan_stage1_ragged", d, "vscan_stage1_ragged_workspace_bytes", workspace)
+    kept_views = [kept[k_off[i]:k_off[i] + k1[i]] for i in range(n)]
+    merged_views = [merged[k_off[i] * D:(k_off[i] + k1[i]) * D].view(k1[i], D) for i in range(n)]
+    return kept_views, merged_views, workspace
+
+
+def vscan_llm_prune_ragged(q_last, k_list, v_list, hidden_list, pos_list, n_sys, n_vis, n_txt, k_keep, scale,
+                           softmax_span=SPAN_ONLY, workspace=None):
+    """Stage 2 for sequences of different lengths in one library call.  q_last [B, Hq, d]; k_list[i], v_list[i]:
+    [Hkv, S_i, d]; hidden_list[i]: [S_i, Dh]; pos_list[i]: [S_i] int32; n_sys .. k_keep: per-sequence lists.
+    Returns a list of dicts (kept_vis, hidden, k, v, pos) of views into the packed outputs, plus the workspace."""
+    B, Hq, d_ = q_last.shape
+    Hkv, Dh = k_list[0].shape[0], hidden_list[0].shape[1]
+    dt, dev = k_list[0].dtype, k_list[0].device
+    e_align = 16 // k_list[0].element_size()
+    S = [a + b + c for a, b, c in zip(n_sys, n_vis, n_txt)]
+    So = [s - b + kk for s, b, kk in zip(S, n_vis, k_keep)]
+    kv_off, kv_total = _aligned_offsets([Hkv * s * d_ for s in S], e_align)
+    kvo_off, kvo_total = _aligned_offsets([Hkv * s * d_ for s in So], e_align)
+    h_off, h_total = _aligned_offsets([s * Dh for s in S], e_align)
+    ho_off, ho_total = _aligned_offsets([s * Dh for s in So], e_align)
+    p_off, p_total = _aligned_offsets(S, 4)
+    po_off, po_total = _aligned_offsets(So, 4)
+    kp_off, kp_total = _aligned_offsets(k_keep, 4)
+    k = torch.zeros(kv_total, dtype=dt, device=dev); v = torch.zeros(kv_total, dtype=dt, device=dev)
+    hidden = torch.zeros(h_total, dtype=dt, device=dev); pos = torch.zeros(p_total, dtype=torch.int32, device=dev)
+    for i in range(B):
+        k[kv_off[i]:kv_off[i] + k_list[i].numel()] = k_list[i].reshape(-1)
+        v[kv_off[i]:kv_off[i] + v_list[i].numel()] = v_list[i].reshape(-1)
+        hidden[h_off[i]:h_off[i] + hidden_list[i].numel()] = hidden_list[i].reshape(-1)
+        pos[p_off[i]:p_off[i] + S[i]] = pos_list[i]
+    k_out = torch.zeros(max(kvo_total, 1), dtype=dt, device=dev); v_out = torch.zeros(max(kvo_total, 1), dtype=dt, device=dev)
+    h_out = torch.zeros(max(ho_total, 1), dtype=dt, device=dev); pos_out = torch.zeros(max(po_total, 1), dtype=torch.int32, device=dev)
+    kept = torch.full((max(kp_total, 1),), -1, dtype=torch.int32, device=dev)
+    keep_alive = [_host_i32(n_sys), _host_i32(n_vis), _host_i32(n_txt), _host_i32(k_keep), _host_i64(kv_off),
+                  _host_i64(kvo_off), _host_i64(h_off), _host_i64(ho_off), _host_i64(p_off), _host_i64(po_off),
+                  _host_i64(kp_off)]
+    desc = PruneRaggedDesc(dtype=_dtype_code(k), batch=B, q_heads=Hq, kv_heads=Hkv, head_dim=d_, hidden_dim=Dh,
+                           pos_planes=1, softmax_span=softmax_span, scale=scale, q_last=_ptr(q_last), k=_ptr(k), v=_ptr(v),
+                           hidden=_ptr(hidden), pos_ids=_ptr(pos), kept_vis=_ptr(kept), hidden_out=_ptr(h_out),
+                           k_out=_ptr(k_out), v_out=_ptr(v_out), pos_out=_ptr(pos_out), n_sys=keep_alive[0],
+                           n_vis=keep_alive[1], n_txt=keep_alive[2], k_keep=keep_alive[3], kv_offset=keep_alive[4],
+                           kv_out_offset=keep_alive[5], hidden_offset=keep_alive[6], hidden_out_offset=keep_alive[7],
+                           pos_offset=keep_alive[8], pos_out_offset=keep_alive[9], kept_offset=keep_alive[10])
+    workspace = _call("vscan_llm_prune_ragged", desc, "vscan_llm_prune_ragged_workspace_bytes", workspace)
+    outs = []
+    for i in range(B):
+        outs.append({"kept_vis": kept[kp_off[i]:kp_off[i] + k_keep[i]],
+                     "k": k_out[kvo_off[i]:kvo_off[i] + Hkv * So[i] * d_].view(Hkv, So[i], d_),
+                     "v": v_out[kvo_off[i]:kvo_off[i] + Hkv * So[i] * d_].view(Hkv, So[i], d_),
+                     "hidden": h_out[ho_off[i]:ho_off[i] + So[i] * Dh].view(So[i], Dh),
+                     "pos": pos_out[po_off[i]:po_off[i] + So[i]]})
+    return outs, workspace
 
 
 def profile_begin(capacity: int = 4096):

@@ -53,6 +53,10 @@ int main(void) {
   P(vscan_merge_desc, x); P(vscan_merge_desc, instances); P(vscan_merge_desc, n_kept); P(vscan_merge_desc, merged); P(vscan_merge_desc, counts);
   printf("vscan_prune_desc %zu\n", sizeof(vscan_prune_desc));
   P(vscan_prune_desc, q_last); P(vscan_prune_desc, batch); P(vscan_prune_desc, k_keep); P(vscan_prune_desc, scale); P(vscan_prune_desc, kept_vis); P(vscan_prune_desc, scores);
+  printf("vscan_stage1_ragged_desc %zu\n", sizeof(vscan_stage1_ragged_desc));
+  P(vscan_stage1_ragged_desc, attn_global); P(vscan_stage1_ragged_desc, merged); P(vscan_stage1_ragged_desc, frames); P(vscan_stage1_ragged_desc, kept_offset);
+  printf("vscan_prune_ragged_desc %zu\n", sizeof(vscan_prune_ragged_desc));
+  P(vscan_prune_ragged_desc, scale); P(vscan_prune_ragged_desc, q_last); P(vscan_prune_ragged_desc, pos_out); P(vscan_prune_ragged_desc, n_sys); P(vscan_prune_ragged_desc, kept_offset);
   return 0;
 }'''
     with tempfile.TemporaryDirectory() as td:
@@ -62,7 +66,8 @@ int main(void) {
         out = subprocess.run([exe], capture_output=True, text=True, check=True).stdout
     got = dict(line.rsplit(" ", 1) for line in out.strip().splitlines())
     structs = {"vscan_score_desc": vb.ScoreDesc, "vscan_select_desc": vb.SelectDesc,
-               "vscan_merge_desc": vb.MergeDesc, "vscan_prune_desc": vb.PruneDesc}
+               "vscan_merge_desc": vb.MergeDesc, "vscan_prune_desc": vb.PruneDesc,
+               "vscan_stage1_ragged_desc": vb.Stage1RaggedDesc, "vscan_prune_ragged_desc": vb.PruneRaggedDesc}
     for key, val in got.items():
         if "." in key:
             s, f = key.split(".")
@@ -165,6 +170,34 @@ def test_merge_and_prune_validation_is_host_side(L):
     p.v = None
     p.n_vis, p.k_keep = 20000, 4
     assert L.vscan_llm_prune(C.byref(p), None, 0, None) == vb.ERR_UNSUPPORTED
+
+
+def test_ragged_validation_is_host_side(L):
+    """Sizes, budgets and offsets of a ragged call are host arrays: everything is checked before a launch."""
+    def stage1(**kw):
+        n = 2
+        base = dict(dtype=vb.BF16, merge_path=vb.MERGE_AUTO, instances=n, heads=4, cls_offset=1, dim=64, win_h=2, win_w=2,
+                    attn_global=FAKE, attn_local=FAKE, x=FAKE + 0x100000, kept_idx=FAKE + 0x200000, merged=FAKE + 0x300000,
+                    frames=[1, 1], grid_h=[4, 6], grid_w=[4, 6], k_per_window=[1, 1], k_global=[2, 2],
+                    attn_offset=[0, 72], x_offset=[0, 17 * 64], kept_offset=[0, 8])
+        base.update(kw)
+        arrays = {k: (vb._host_i64(v) if k.endswith("offset") else vb._host_i32(v)) for k, v in base.items() if isinstance(v, list)}
+        base.update(arrays)
+        d = vb.Stage1RaggedDesc(**base)
+        return L.vscan_stage1_ragged(C.byref(d), None, 0, None), L.vscan_stage1_ragged_workspace_bytes(C.byref(d))
+    st, need = stage1()
+    assert st == vb.ERR_WORKSPACE and need > 256                 # legal call: next check is the workspace
+    assert stage1(grid_h=[4, 5])[0] == vb.ERR_INVALID_ARG         # window does not divide the second grid
+    assert stage1(attn_offset=[0, 69])[0] == vb.ERR_WORKSPACE     # (alignment is checked after the workspace)
+    assert stage1(instances=0)[0] == vb.OK
+    assert stage1(frames=None)[0] == vb.ERR_INVALID_ARG
+    p = vb.PruneRaggedDesc(dtype=vb.BF16, batch=1, q_heads=4, kv_heads=2, head_dim=32, hidden_dim=0, pos_planes=0, scale=1.0,
+                           q_last=FAKE, k=FAKE + 0x100000, kept_vis=FAKE + 0x200000, k_out=FAKE + 0x300000,
+                           n_sys=vb._host_i32([2]), n_vis=vb._host_i32([8]), n_txt=vb._host_i32([2]), k_keep=vb._host_i32([9]),
+                           kv_offset=vb._host_i64([0]), kv_out_offset=vb._host_i64([0]), kept_offset=vb._host_i64([0]))
+    assert L.vscan_llm_prune_ragged(C.byref(p), None, 0, None) == vb.ERR_INVALID_ARG   # k_keep > n_vis
+    p.k_keep = vb._host_i32([4])
+    assert L.vscan_llm_prune_ragged(C.byref(p), None, 0, None) == vb.ERR_WORKSPACE
 
 
 def test_stale_library_is_rebuilt_or_refused(monkeypatch, tmp_path):
