@@ -440,6 +440,9 @@ def run_sweep(args, rank, world, local_rank, dist):
     if rank == 0 and (not args.sweep_filter or args.sweep_filter in "ragged"):
         import torch
         print(json.dumps(measure_ragged(args, torch.device("cuda", local_rank))), flush=True)
+    if rank == 0 and (not args.sweep_filter or args.sweep_filter in "received"):
+        import torch
+        print(json.dumps(measure_received(args, torch.device("cuda", local_rank), peak_tf)), flush=True)
     for label, cfg, path, s1 in points:
         args.merge_path = path
         steps = args.steps
@@ -459,6 +462,43 @@ def run_sweep(args, rank, world, local_rank, dist):
                "kernels_us": {n: round(v["avg_us"] * v["launches_per_step"], 1) for n, v in k.items()},
                "clocks_mhz": line["clocks"]["sm_mhz"], "reasons": line["clocks"]["reasons"]}
         print(json.dumps(out), flush=True)
+
+
+def measure_received(args, device, peak_tf):
+    """The no-[CLS] score source at the 16384-token shape (4 instances x 16 heads, head dim 128): received
+    attention from q and k in two tensor-core passes over the score matrix, which is never stored."""
+    import torch
+
+    from paper_2505_22654_b200 import binding as vb
+    B, H, N, d = 4, 16, 16384, 128
+    g = torch.Generator(device="cpu").manual_seed(0)
+    q = torch.randn((B, H, N, d), generator=g).to(torch.bfloat16).to(device)
+    k = torch.randn((B, H, N, d), generator=g).to(torch.bfloat16).to(device)
+    out = torch.empty((B, N), dtype=torch.float32, device=device)
+    ws = vb.Workspace(0, device)
+    stream = torch.cuda.Stream(device)
+    with torch.cuda.stream(stream):
+        L = vb.lib()
+        import ctypes as C
+        desc = vb.ScoreDesc(mode=vb.SCORE_RECEIVED, dtype=vb.BF16, q=q.data_ptr(), k=k.data_ptr(), batch=B, q_heads=H,
+                            kv_heads=H, seq_len=N, head_dim=d, scale=d ** -0.5, scores=out.data_ptr())
+        ws.reserve(L.vscan_score_workspace_bytes(C.byref(desc)))
+        vb.vscan_score_received(q, k, d ** -0.5, out=out, workspace=ws)
+        stream.synchronize()
+        n = 3
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            vb.vscan_score_received(q, k, d ** -0.5, out=out, workspace=ws)
+        e1.record(stream)
+        e1.synchronize()
+        status = vb.vscan_check(ws)
+    ms = e0.elapsed_time(e1) / n
+    flops = 2 * 2.0 * B * H * N * N * d
+    return {"point": "received attention from q, k: 4 x 16 heads x 16384 tokens x 128", "ms": round(ms, 3),
+            "tflops": round(flops / (ms * 1e-3) / 1e12, 1), "tensor_frac": round(flops / (ms * 1e-3) / 1e12 / peak_tf, 3),
+            "exp_per_s": round(2.0 * B * H * N * N / (ms * 1e-3) / 1e12, 2), "status": status,
+            "score_sum_per_instance": [round(float(v), 4) for v in out.sum(dim=1).tolist()]}
 
 
 def measure_ragged(args, device):

@@ -51,7 +51,7 @@ typedef enum {
 } vscan_status;
 
 typedef enum { VSCAN_F32 = 0, VSCAN_BF16 = 1 } vscan_dtype;
-typedef enum { VSCAN_SCORE_ROW = 0, VSCAN_SCORE_QK = 1 } vscan_score_mode;
+typedef enum { VSCAN_SCORE_ROW = 0, VSCAN_SCORE_QK = 1, VSCAN_SCORE_RECEIVED = 2 } vscan_score_mode;
 /* Eq. 5 takes the softmax over the visual keys only (SPAN_ONLY); Sec. 4.2's remark on recomputing
  * "vanilla attention" for the last token normalises over all keys (SPAN_FULL). */
 typedef enum { VSCAN_SPAN_ONLY = 0, VSCAN_SPAN_FULL = 1 } vscan_softmax_span;
@@ -84,7 +84,15 @@ typedef enum {
  *   k         [batch][kv_heads][seq_len][head_dim] of `dtype`
  *   scores    [batch][span_len] float32 (output).  head_dim must be a multiple of 8, at most 256;
  *             q_heads a multiple of kv_heads.
- * Fields of the mode not in use are ignored.  Workspace: QK mode only.
+ * RECEIVED mode (Sec. 4.1, text after Eq. 2: encoders without [CLS] score a token by the average attention it
+ *   receives from the other tokens): with P_h = softmax over keys of (scale * q[b][h] k[b][h]^T), row by row,
+ *   r_h[j] = (1 / (seq_len - 1)) * sum_{i != j} P_h[i][j];  scores[b][j] = (1/q_heads) * sum_h r_h[j].
+ *   The seq_len x seq_len matrix is never stored: two passes over 128 x 128 blocks on the tensor cores.
+ *   q, k      [batch][q_heads][seq_len][head_dim] of `dtype` (kv_heads must equal q_heads)
+ *   scores    [batch][seq_len] float32 (output)
+ *   head_rows optional [batch][q_heads][seq_len] float32 output: the per-head r_h (what ROW mode takes as `attn`)
+ *   This build: VSCAN_BF16 with head_dim 64 or 128, batch * q_heads <= 65535; else VSCAN_ERR_UNSUPPORTED.
+ * Fields of the mode not in use are ignored.  Workspace: QK and RECEIVED modes.
  * Limits of this build (VSCAN_ERR_UNSUPPORTED, nothing enqueued): instances, batch <= 65535; QK mode:
  * (head_dim + keys under the softmax) * 4 bytes must fit 227 KB of shared memory (about 58 000 keys).
  * ------------------------------------------------------------------------------------------- */
@@ -102,6 +110,7 @@ typedef struct {
   float scale;
   /* output */
   float* scores;
+  float* head_rows; /* RECEIVED mode, optional */
 } vscan_score_desc;
 
 size_t vscan_score_workspace_bytes(const vscan_score_desc* desc);

@@ -15,7 +15,7 @@ from . import _build
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 F32, BF16 = 0, 1
-SCORE_ROW, SCORE_QK = 0, 1
+SCORE_ROW, SCORE_QK, SCORE_RECEIVED = 0, 1, 2
 SPAN_ONLY, SPAN_FULL = 0, 1
 MERGE_AUTO, MERGE_SIMT, MERGE_TENSOR, MERGE_INTERLEAVED = 0, 1, 2, 4
 
@@ -27,7 +27,7 @@ class ScoreDesc(C.Structure):
                 ("row_len", _i32), ("cls_offset", _i32), ("n_tokens", _i32), ("q", _vp), ("k", _vp),
                 ("batch", _i32), ("q_heads", _i32), ("kv_heads", _i32), ("seq_len", _i32),
                 ("head_dim", _i32), ("span_begin", _i32), ("span_len", _i32), ("softmax_span", _i32),
-                ("scale", _f32), ("scores", _vp)]
+                ("scale", _f32), ("scores", _vp), ("head_rows", _vp)]
 
 
 class SelectDesc(C.Structure):
@@ -230,6 +230,19 @@ def vscan_score_qk(q, k, span_begin, span_len, scale, softmax_span=SPAN_ONLY, ou
     d = score_qk_desc(q, k, span_begin, span_len, scale, softmax_span, out)
     _call("vscan_score", d, "vscan_score_workspace_bytes", workspace)
     return out
+
+
+def vscan_score_received(q, k, scale, out=None, want_head_rows=False, workspace=None):
+    """Sec. 4.1 (text after Eq. 2): head mean of the attention every token receives from the others, from
+    q, k [B', H, N, d] without the N x N matrix.  -> scores [B', N] float32 (and the per-head rows [B', H, N])."""
+    B, H, N, d = q.shape
+    if out is None:
+        out = torch.empty((B, N), dtype=torch.float32, device=q.device)
+    rows = torch.empty((B, H, N), dtype=torch.float32, device=q.device) if want_head_rows else None
+    desc = ScoreDesc(mode=SCORE_RECEIVED, dtype=_dtype_code(q), q=_ptr(q), k=_ptr(k), batch=B, q_heads=H, kv_heads=H,
+                     seq_len=N, head_dim=d, scale=scale, scores=_ptr(out), head_rows=_ptr(rows))
+    _call("vscan_score", desc, "vscan_score_workspace_bytes", workspace)
+    return (out, rows) if want_head_rows else out
 
 
 def vscan_score_qk_static(q, k, span_begin, span_len, scale, out, softmax_span=SPAN_ONLY):

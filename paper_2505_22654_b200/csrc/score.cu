@@ -93,6 +93,20 @@ vscan_status validate_score(const vscan_score_desc* d) {
       return VSCAN_ERR_INVALID_ARG;
     return VSCAN_OK;
   }
+  if (d->mode == VSCAN_SCORE_RECEIVED) {
+    if (!d->q || !d->k || !aligned16(d->q) || !aligned16(d->k)) return VSCAN_ERR_INVALID_ARG;
+    if (d->head_rows && !aligned16(d->head_rows)) return VSCAN_ERR_INVALID_ARG;
+    if (d->batch < 0 || d->q_heads <= 0 || d->kv_heads != d->q_heads || d->seq_len <= 0 || d->head_dim <= 0 || d->head_dim % 8)
+      return VSCAN_ERR_INVALID_ARG;
+    if (1ll * d->batch * d->q_heads > 65535) return VSCAN_ERR_UNSUPPORTED;
+    if (!received_supported(d)) return VSCAN_ERR_UNSUPPORTED;   // bf16, head_dim 64 or 128
+    const size_t qk = static_cast<size_t>(d->batch) * d->q_heads * d->seq_len * d->head_dim * e;
+    const size_t rows = static_cast<size_t>(d->batch) * d->q_heads * d->seq_len * 4, sc = static_cast<size_t>(d->batch) * d->seq_len * 4;
+    if (overlaps(d->scores, sc, d->q, qk) || overlaps(d->scores, sc, d->k, qk) || overlaps(d->head_rows, rows, d->q, qk) ||
+        overlaps(d->head_rows, rows, d->k, qk) || overlaps(d->head_rows, rows, d->scores, sc))
+      return VSCAN_ERR_INVALID_ARG;
+    return VSCAN_OK;
+  }
   return VSCAN_ERR_INVALID_ARG;
 }
 
@@ -101,6 +115,7 @@ vscan_status validate_score(const vscan_score_desc* d) {
 using namespace vscan;
 
 extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
+  if (d && d->mode == VSCAN_SCORE_RECEIVED && d->batch > 0 && d->q_heads > 0 && d->seq_len > 0) return received_workspace_bytes(d);
   if (!d || d->mode != VSCAN_SCORE_QK || d->batch <= 0 || d->q_heads <= 0 || d->span_len <= 0) return 0;
   return kStatusBytes + round_up(static_cast<size_t>(d->batch) * sizeof(int), 256) +
          round_up(static_cast<size_t>(d->batch) * d->q_heads * d->span_len * sizeof(float), 256);
@@ -108,7 +123,7 @@ extern "C" size_t vscan_score_workspace_bytes(const vscan_score_desc* d) {
 
 extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, size_t workspace_bytes,
                                     void* stream_) {
-  if (d && ((d->mode == VSCAN_SCORE_ROW && d->instances == 0) || (d->mode == VSCAN_SCORE_QK && d->batch == 0)))
+  if (d && ((d->mode == VSCAN_SCORE_ROW && d->instances == 0) || ((d->mode == VSCAN_SCORE_QK || d->mode == VSCAN_SCORE_RECEIVED) && d->batch == 0)))
     return VSCAN_OK;  // empty batch: nothing to read or write
   vscan_status st = validate_score(d);
   if (st != VSCAN_OK) return st;
@@ -125,6 +140,21 @@ extern "C" vscan_status vscan_score(const vscan_score_desc* d, void* workspace, 
                    row_mean_kernel<__nv_bfloat16><<<grid, 256, 0, stream>>>(
                        static_cast<const __nv_bfloat16*>(d->attn), d->scores, d->heads, d->row_len, d->cls_offset,
                        d->n_tokens));
+    return VSCAN_OK;
+  }
+  if (d->mode == VSCAN_SCORE_RECEIVED) {
+    const size_t need = vscan_score_workspace_bytes(d);
+    if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
+    const size_t bh = static_cast<size_t>(d->batch) * d->q_heads;
+    float* rows = d->head_rows ? d->head_rows
+                               : reinterpret_cast<float*>(static_cast<char*>(workspace) + kStatusBytes +
+                                                          round_up(bh * round_up(d->seq_len, 128) * sizeof(float), 256));
+    st = launch_received(d, workspace, rows, stream);
+    if (st != VSCAN_OK) return st;
+    // Eq. 2 on the per-head rows
+    dim3 grid((d->seq_len + 255) / 256, d->batch);
+    VSCAN_LAUNCH("row_mean", stream,
+                 row_mean_kernel<float><<<grid, 256, 0, stream>>>(rows, d->scores, d->q_heads, d->seq_len, 0, d->seq_len));
     return VSCAN_OK;
   }
   if (d->batch == 0 || d->span_len == 0) return VSCAN_OK;

@@ -190,5 +190,9 @@ inline size_t qk_smem_bytes(int head_dim, int soft_n) {
 // Host-side argument checks and launch shared by the entry points.
 vscan_status validate_score(const vscan_score_desc* d);
 vscan_status launch_qk_softmax(int dtype, const QkParams& p, int batch, cudaStream_t stream);
+// RECEIVED mode (Sec. 4.1, text after Eq. 2): per-head received attention from Q and K on the tensor cores.
+bool received_supported(const vscan_score_desc* d);
+size_t received_workspace_bytes(const vscan_score_desc* d);
+vscan_status launch_received(const vscan_score_desc* d, void* workspace, float* rows_out, cudaStream_t stream);
 
 }  // namespace vscan

@@ -46,7 +46,7 @@ def test_struct_layout_matches_header():
 #define P(s, f) printf(#s "." #f " %zu\n", offsetof(s, f))
 int main(void) {
   printf("vscan_score_desc %zu\n", sizeof(vscan_score_desc));
-  P(vscan_score_desc, attn); P(vscan_score_desc, q); P(vscan_score_desc, batch); P(vscan_score_desc, scale); P(vscan_score_desc, scores);
+  P(vscan_score_desc, attn); P(vscan_score_desc, q); P(vscan_score_desc, batch); P(vscan_score_desc, scale); P(vscan_score_desc, scores); P(vscan_score_desc, head_rows);
   printf("vscan_select_desc %zu\n", sizeof(vscan_select_desc));
   P(vscan_select_desc, instances); P(vscan_select_desc, kept_idx); P(vscan_select_desc, kept_mask);
   printf("vscan_merge_desc %zu\n", sizeof(vscan_merge_desc));
@@ -121,6 +121,23 @@ def test_score_validation_is_host_side(L):
     assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG
     assert L.vscan_score_qk_static(C.byref(d), None) == vb.ERR_INVALID_ARG    # same checks in the static variant
     d.scores = FAKE + 0x800000
+
+
+def test_received_mode_validation(L):
+    d = vb.ScoreDesc(mode=vb.SCORE_RECEIVED, dtype=vb.BF16, q=FAKE, k=FAKE + 0x1000000, batch=2, q_heads=4, kv_heads=4,
+                     seq_len=300, head_dim=64, scale=0.125, scores=FAKE + 0x2000000)
+    assert L.vscan_score_workspace_bytes(C.byref(d)) >= 256 + 8 * 384 * 4 + 8 * 300 * 4
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_WORKSPACE        # legal: next check is the workspace
+    d.kv_heads = 2
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG      # every head has its own keys here
+    d.kv_heads, d.head_dim = 4, 80
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_UNSUPPORTED      # head_dim 64 or 128 in this build
+    d.head_dim, d.dtype = 64, vb.F32
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_UNSUPPORTED      # tensor-core path: bf16 only
+    d.dtype, d.batch = vb.BF16, 20000
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_UNSUPPORTED      # batch * heads beyond the grid limit
+    d.batch, d.scores = 2, FAKE
+    assert L.vscan_score(C.byref(d), None, 0, None) == vb.ERR_INVALID_ARG      # output on top of q
 
 
 def test_shape_limits_are_refused_before_anything_is_enqueued(L):

@@ -315,6 +315,48 @@ def test_cls_scores_from_q_and_k_eq1_eq2(dtype):
         assert abs(alt[b].sum() - 1.0) < 1e-5
 
 
+@pytest.mark.parametrize("B,H,N,d", [(2, 3, 300, 64), (1, 4, 2048, 128), (1, 2, 129, 64), (3, 1, 128, 128), (2, 2, 1, 64)])
+def test_received_attention_scores_from_q_and_k(B, H, N, d):
+    """Sec. 4.1 (text after Eq. 2): for encoders without [CLS] the score of a token is the head mean of the average
+    attention it receives from the other tokens.  The library computes it from q and k block by block; the oracle
+    builds every head's full softmax matrix in float64 and takes its column means without the diagonal.  Tolerance:
+    the scores are means of probabilities (<= 1) accumulated in fp32 from base-2 exponentials whose argument carries
+    a relative rounding error of 2^-24 on values of up to a few tens: relative error of a probability about 2e-6,
+    far below the 2e-6 absolute bar for values of the order 1/N."""
+    rng = np.random.default_rng(N + d)
+    q = round_to_dtype(rng.standard_normal((B, H, N, d)).astype(np.float32), "bf16")
+    k = round_to_dtype(rng.standard_normal((B, H, N, d)).astype(np.float32), "bf16")
+    scale = float(d ** -0.5)
+    ws = vs.Workspace(0)
+    got, rows = vs.vscan_score_received(dev(q, "bf16"), dev(k, "bf16"), scale, want_head_rows=True, workspace=None)
+    got, rows = got.cpu().numpy(), rows.cpu().numpy()
+    for b in range(B):
+        z = scale * np.einsum("hid,hjd->hij", q[b].astype(np.float64), k[b].astype(np.float64))
+        z -= z.max(axis=2, keepdims=True)
+        p = np.exp(z)
+        p /= p.sum(axis=2, keepdims=True)
+        ref_rows = vo.received_attention(p)
+        assert np.abs(rows[b] - ref_rows).max() <= TOL_SCORE
+        assert np.abs(got[b] - vo.score_row(ref_rows, 0)).max() <= TOL_SCORE
+    if N > 1:   # every query's attention sums to one, so the received attention sums to (N - diag mass) / (N - 1) <= N / (N - 1)
+        assert np.all(got.sum(axis=1) <= N / (N - 1) + 1e-4)
+    del ws
+
+
+def test_received_attention_feeds_the_selection():
+    """The received-attention scores go straight into the selection (the 16384-token workload without handed-in rows,
+    at a size the oracle can follow): kept indices equal the oracle's on the library's own fp32 scores."""
+    rng = np.random.default_rng(5)
+    B, H, N, d = 2, 4, 1024, 64
+    q = round_to_dtype(rng.standard_normal((B, H, N, d)).astype(np.float32), "bf16")
+    k = round_to_dtype(rng.standard_normal((B, H, N, d)).astype(np.float32), "bf16")
+    s = vs.vscan_score_received(dev(q, "bf16"), dev(k, "bf16"), float(d ** -0.5))
+    kept = vs.vscan_select_global_local(s, s, 1, 32, 32, 8, 8, 2, 64).cpu().numpy()
+    s32 = s.cpu().numpy()
+    for b in range(B):
+        np.testing.assert_array_equal(kept[b], vo.select_global_local(s32[b], s32[b], 1, 32, 32, 8, 8, 2, 64)[0])
+
+
 # ------------------------------------------------------------------ vscan_llm_prune
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("span", [vo.SPAN_ONLY, vo.SPAN_FULL])
