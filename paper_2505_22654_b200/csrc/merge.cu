@@ -166,6 +166,181 @@ __global__ void __launch_bounds__(128) group_mean_bits_kernel(MergeParams p) {
   group_mean_bits_body<T, VPL, R>(p, blockIdx.y, blockIdx.x * 4, smem_bits);
 }
 
+// ---- long instances (more than 2048 tokens): members by counting sort, segments put in order, then the sums.
+// order_kernel, one CTA per instance: histogram of the assignments over the kept slots (shared-memory atomics),
+// exclusive scan -> start[instance][n_kept + 1], then every token is dropped into its slot's segment of
+// order[instance][n_tokens] (segment cursors are shared-memory atomics, so the order inside a segment is arbitrary).
+__global__ void __launch_bounds__(1024) order_kernel(MergeParams p, int32_t* order, int32_t* start) {
+  extern __shared__ __align__(16) int hist[];          // n_kept + 1 cursors
+  __shared__ int warp_sums[33];
+  grid_dependency_wait();                               // the assignments come from the kernel before this one
+  const int b = blockIdx.x;
+  const int32_t* ag = p.assign + static_cast<size_t>(b) * p.n_tokens;
+  for (int s = threadIdx.x; s <= p.n_kept; s += blockDim.x) hist[s] = 0;
+  __syncthreads();
+  for (int i = threadIdx.x; i < p.n_tokens; i += blockDim.x) atomicAdd(&hist[min(max(__ldcg(ag + i), 0), p.n_kept - 1)], 1);
+  __syncthreads();
+  // exclusive scan of the n_kept counts, a contiguous run of slots per thread
+  const int per = (p.n_kept + blockDim.x - 1) / blockDim.x;
+  const int lo = min(p.n_kept, static_cast<int>(threadIdx.x) * per), hi = min(p.n_kept, lo + per);
+  int mine = 0;
+  for (int s = lo; s < hi; ++s) mine += hist[s];
+  int total;
+  int run = block_exclusive_scan(mine, warp_sums, total);
+  int32_t* st = start + static_cast<size_t>(b) * (p.n_kept + 1);
+  for (int s = lo; s < hi; ++s) { const int c = hist[s]; hist[s] = run; st[s] = run; run += c; }
+  if (threadIdx.x == 0) st[p.n_kept] = total;
+  __syncthreads();
+  int32_t* od = order + static_cast<size_t>(b) * p.n_tokens;
+  for (int i = threadIdx.x; i < p.n_tokens; i += blockDim.x) od[atomicAdd(&hist[min(max(__ldcg(ag + i), 0), p.n_kept - 1)], 1)] = i;
+}
+
+// sort_segments_kernel: one warp per kept slot puts its segment of `order` into ascending token order, in place:
+// up to 32 members by rank counting in registers, up to kSortMax by a bitonic network in the warp's shared memory,
+// beyond that (one slot holding thousands of tokens) by repeated minimum search.
+constexpr int kSortMax = 2048;
+__global__ void __launch_bounds__(256) sort_segments_kernel(MergeParams p, int32_t* order, const int32_t* start) {
+  extern __shared__ __align__(16) int32_t sort_all[];
+  grid_dependency_wait();
+  const int b = blockIdx.y, w = threadIdx.x >> 5, lane = threadIdx.x & 31, s = blockIdx.x * 8 + w;
+  if (s >= p.n_kept) return;
+  const int32_t* st = start + static_cast<size_t>(b) * (p.n_kept + 1);
+  const int seg0 = __ldcg(st + s), count = __ldcg(st + s + 1) - seg0;
+  int32_t* seg = order + static_cast<size_t>(b) * p.n_tokens + seg0;
+  if (count <= 1) return;
+  if (count <= 32) {
+    const int mine = lane < count ? __ldcg(seg + lane) : 0x7fffffff;
+    int rank = 0;
+#pragma unroll
+    for (int l = 0; l < 32; ++l) rank += __shfl_sync(0xffffffffu, mine, l) < mine;   // ids are distinct
+    if (lane < count) seg[rank] = mine;
+    return;
+  }
+  if (count <= kSortMax) {
+    int32_t* a = sort_all + w * kSortMax;
+    int n = 64;
+    while (n < count) n <<= 1;
+    for (int i = lane; i < n; i += 32) a[i] = i < count ? __ldcg(seg + i) : 0x7fffffff;
+    __syncwarp();
+    for (int k = 2; k <= n; k <<= 1)
+      for (int jj = k >> 1; jj > 0; jj >>= 1) {
+        for (int idx = lane; idx < n / 2; idx += 32) {
+          const int l = ((idx / jj) * 2 * jj) + (idx % jj), r = l + jj;
+          const int x = a[l], y = a[r];
+          const bool up = (l & k) == 0;
+          if ((x > y) == up) { a[l] = y; a[r] = x; }
+        }
+        __syncwarp();
+      }
+    for (int i = lane; i < count; i += 32) seg[i] = a[i];
+    return;
+  }
+  // oversized segment: selection sort with warp-wide minimum search (quadratic, for the pathological case only)
+  for (int k = 0; k < count - 1; ++k) {
+    int best = 0x7fffffff, at = -1;
+    for (int i = k + lane; i < count; i += 32) { const int t = seg[i]; if (t < best) { best = t; at = i; } }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const int ob = __shfl_xor_sync(0xffffffffu, best, o), oa = __shfl_xor_sync(0xffffffffu, at, o);
+      if (ob < best) { best = ob; at = oa; }
+    }
+    if (lane == 0 && at != k) { const int t = seg[k]; seg[k] = best; seg[at] = t; }
+    __syncwarp();
+  }
+}
+
+// group_mean_sorted_kernel: one warp per (kept slot, chunk of 32 * VPL 16-byte column pieces).  The warp walks the
+// slot's ordered segment and adds the rows' chunk in that order, R rows in flight: the same additions in the same
+// order as the other CUDA-core group means.  Splitting the columns over warps keeps a slot with hundreds of members
+// from becoming one long chain.
+template <typename T, int VPL, int R>
+__global__ void __launch_bounds__(256) group_mean_sorted_kernel(MergeParams p, const int32_t* order, const int32_t* start, int chunks) {
+  constexpr int E = Vec16<T>::kElems;
+  grid_dependency_wait();
+  const int b = blockIdx.y, lane = threadIdx.x & 31;
+  const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
+  const int s = task / chunks, v0 = (task - s * chunks) * 32 * VPL;
+  if (s >= p.n_kept) return;
+  const int32_t* st = start + static_cast<size_t>(b) * (p.n_kept + 1);
+  const int seg0 = __ldcg(st + s), count = __ldcg(st + s + 1) - seg0;
+  const int32_t* seg = order + static_cast<size_t>(b) * p.n_tokens + seg0;
+  const int vecs = p.dim / E;
+  const T* xb = static_cast<const T*>(p.x) + (static_cast<size_t>(b) * p.row_len + p.cls_offset) * p.dim;
+  T* out = static_cast<T*>(p.merged) + (static_cast<size_t>(b) * p.n_kept + s) * p.dim;
+  float acc[VPL][E];
+#pragma unroll
+  for (int i = 0; i < VPL; ++i)
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[i][e] = 0.f;
+  for (int k0 = 0; k0 < count; k0 += 32) {
+    const int mine = k0 + lane < count ? min(max(__ldcg(seg + k0 + lane), 0), p.n_tokens - 1) : -1;   // 32 members per round of ids
+    const int here = min(32, count - k0);
+    for (int k = 0; k < here; k += R) {
+      uint4 raw[R][VPL];
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int tok = __shfl_sync(0xffffffffu, mine, min(k + r, 31));
+        if (k + r < here) {
+          const uint4* row = reinterpret_cast<const uint4*>(xb + static_cast<size_t>(tok) * p.dim);
+#pragma unroll
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs) raw[r][i] = ld_nc_16(row + v);
+          }
+        }
+      }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        if (k + r < here) {
+#pragma unroll
+          for (int i = 0; i < VPL; ++i) {
+            const int v = v0 + lane + 32 * i;
+            if (v < vecs) {
+              float f[E];
+              Vec16<T>::unpack(raw[r][i], f);
+#pragma unroll
+              for (int e = 0; e < E; ++e) acc[i][e] += f[e];
+            }
+          }
+        }
+      }
+    }
+  }
+  const float inv = 1.f / static_cast<float>(max(count, 1));
+#pragma unroll
+  for (int i = 0; i < VPL; ++i) {
+    const int v = v0 + lane + 32 * i;
+    if (v < vecs) {
+      float f[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) f[e] = acc[i][e] * inv;
+      st_16(reinterpret_cast<uint4*>(out) + v, Vec16<T>::pack(f));
+    }
+  }
+  if (v0 == 0 && lane == 0 && p.counts) p.counts[static_cast<size_t>(b) * p.n_kept + s] = count;
+}
+
+template <typename T>
+static vscan_status launch_group_mean_sorted(const MergeParams& p, cudaStream_t stream) {
+  constexpr int E = Vec16<T>::kElems, VPL = 1, R = 8;
+  const size_t smem_order = (static_cast<size_t>(p.n_kept) + 1) * sizeof(int);
+  VSCAN_CUDA_TRY(allow_smem(order_kernel, smem_order));
+  VSCAN_LAUNCH("order_members", stream,
+               (void)launch_dependent(order_kernel, dim3(p.instances), dim3(1024), smem_order, stream, p, p.order, p.order_start));
+  const size_t smem_sort = 8 * kSortMax * sizeof(int32_t);
+  VSCAN_CUDA_TRY(allow_smem(sort_segments_kernel, smem_sort));
+  dim3 sgrid((p.n_kept + 7) / 8, p.instances);
+  VSCAN_LAUNCH("order_members", stream,
+               (void)launch_dependent(sort_segments_kernel, sgrid, dim3(256), smem_sort, stream, p, p.order,
+                                      static_cast<const int32_t*>(p.order_start)));
+  const int chunks = (p.dim / E + 32 * VPL - 1) / (32 * VPL);
+  dim3 grid((static_cast<unsigned>(p.n_kept) * chunks + 7) / 8, p.instances);
+  VSCAN_LAUNCH("group_mean", stream,
+               (void)launch_dependent(group_mean_sorted_kernel<T, VPL, R>, grid, dim3(256), 0, stream, p,
+                                      static_cast<const int32_t*>(p.order), static_cast<const int32_t*>(p.order_start), chunks));
+  return VSCAN_OK;
+}
+
 template <typename T, int VPL, int R>
 static vscan_status launch_group_mean_bits(const MergeParams& p, cudaStream_t stream) {
   const size_t chunks = (static_cast<size_t>(p.n_tokens) + 31) / 32;
@@ -194,6 +369,9 @@ static vscan_status launch_group_mean(const MergeParams& p, cudaStream_t stream)
   const bool wide = p.dim / E > 128, long_instance = p.n_tokens > 2048;
   // 512-thread CTAs have 128 registers per thread: wide rows are then summed in two column passes
   // (4 pieces per lane each) rather than with 8 pieces per lane, which would spill
+  // long instances: counting sort + one warp per slot while groups are small on average (each warp orders its
+  // own members); with few slots the groups are long lists, which the CTA-wide ordered listing handles better
+  if (long_instance && static_cast<long long>(p.n_kept) * 64 >= p.n_tokens && p.order) return launch_group_mean_sorted<T>(p, stream);
   if (long_instance) return launch_group_mean_as<T, 4, 4, 16>(p, smem, stream);
   if (!wide) return launch_group_mean_bits<T, 2, 4>(p, stream);   // two column passes, few registers: more CTAs per SM
   return launch_group_mean_as<T, 8, 2, 4>(p, smem, stream);
@@ -244,6 +422,10 @@ extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
   size_t bytes = kStatusBytes;
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256);    // inv_norm
   bytes += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);  // assign
+  if (d->n_tokens > 2048) {   // long instances: tokens ordered by slot, segment starts
+    bytes += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);
+    bytes += round_up(static_cast<size_t>(d->instances) * (static_cast<size_t>(d->n_kept) + 1) * sizeof(int32_t), 256);
+  }
   if (d->dtype == VSCAN_BF16) {   // packed copy of the kept rows for the tensor paths
     const size_t md = d->metric ? d->metric_dim : d->dim;
     bytes += round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * md * 2, 256);
@@ -273,10 +455,15 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   int32_t* ws_assign = reinterpret_cast<int32_t*>(
       ws + kStatusBytes + round_up(static_cast<size_t>(d->instances) * d->n_kept * sizeof(float), 256));
   p.assign = d->assign ? d->assign : ws_assign;
-  p.kept_packed = d->dtype == VSCAN_BF16
-                      ? static_cast<void*>(reinterpret_cast<char*>(ws_assign) +
-                                           round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256))
-                      : nullptr;
+  char* ws_next = reinterpret_cast<char*>(ws_assign) + round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);
+  p.order = nullptr; p.order_start = nullptr;
+  if (d->n_tokens > 2048) {
+    p.order = reinterpret_cast<int32_t*>(ws_next);
+    ws_next += round_up(static_cast<size_t>(d->instances) * d->n_tokens * sizeof(int32_t), 256);
+    p.order_start = reinterpret_cast<int32_t*>(ws_next);
+    ws_next += round_up(static_cast<size_t>(d->instances) * (static_cast<size_t>(d->n_kept) + 1) * sizeof(int32_t), 256);
+  }
+  p.kept_packed = d->dtype == VSCAN_BF16 ? static_cast<void*>(ws_next) : nullptr;
   p.counters = p.kept_packed ? reinterpret_cast<int*>(static_cast<char*>(p.kept_packed) +
                                                       round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * p.metric_dim * 2, 256))
                              : nullptr;

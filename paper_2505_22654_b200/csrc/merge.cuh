@@ -16,6 +16,8 @@ struct MergeParams {
   void* kept_packed;    // [instances][n_kept rounded up to 256, or to 16 when <= 256][metric_dim] copy of the kept rows   (workspace;
                         // only for kept sets above 256, where it feeds the tensor path with plain tile loads)
   int* counters;        // [instances + 1] counters of the persistent path                              (workspace)
+  int32_t* order;       // [instances][n_tokens] tokens ordered by slot, long instances only            (workspace)
+  int32_t* order_start; // [instances][n_kept + 1] segment starts of `order`                            (workspace)
   int clear_status;     // this launch resets the status word (first launch of a call)
   uint32_t* status;     // device status word
   int instances, row_len, cls_offset, n_tokens, dim, metric_dim, n_kept;

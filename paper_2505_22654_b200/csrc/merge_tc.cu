@@ -32,6 +32,7 @@ struct Params {
   int stages;
   int tmem_cols;    // power of two >= max(32, n_pad)
   int a_stage_bytes, b_stage_bytes;
+  int norms_given;  // 1 / |m_s| comes from the packing kernel (m.inv_norm) instead of being taken from the B stages
 };
 
 struct Shared {
@@ -43,24 +44,6 @@ struct Shared {
   int abort_flag;
   int best_slot[kTileM];
 };
-
-// Copies the kept rows of every instance into a contiguous [instance][slot][dim] buffer (slots past
-// n_kept are zero).  One warp per slot.
-__global__ void __launch_bounds__(256) pack_kept_kernel(MergeParams m, int rows_packed) {
-  const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-  if (s >= rows_packed) return;
-  uint4* dst = reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(m.kept_packed) +
-                                        (static_cast<size_t>(b) * rows_packed + s) * m.metric_dim);
-  const int vecs = m.metric_dim / 8;
-  if (s < m.n_kept) {
-    const int t = min(max(m.kept[static_cast<size_t>(b) * m.n_kept + s], 0), m.n_tokens - 1);
-    const uint4* src = reinterpret_cast<const uint4*>(
-        static_cast<const __nv_bfloat16*>(m.metric) + (static_cast<size_t>(b) * m.row_len + m.cls_offset + t) * m.metric_dim);
-    for (int v = lane; v < vecs; v += 32) st_16(dst + v, ld_nc_16(src + v));
-  } else {
-    for (int v = lane; v < vecs; v += 32) st_16(dst + v, make_uint4(0u, 0u, 0u, 0u));
-  }
-}
 
 // The whole life of one assignment CTA: tile of 128 tokens starting at token t0 of instance b.
 // smem_dyn: up to 1023 bytes of alignment slack | stages x [A tile 128x64 bf16 | B tile n_pad x 64 bf16] |
@@ -83,7 +66,8 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
   if (threadIdx.x == 0) {
     // a stage is free again once the MMAs that read it have completed and the four epilogue warps
     // have taken the squared norms of its kept-row slice
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 5); }
+    // (with norms from the packing kernel the read-back warps never touch the stages)
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], p.norms_given ? 1 : 5); }
     for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 4); }
     sh.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -97,7 +81,7 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = sh.tmem_base;
   grid_dependency_launch();
-  grid_dependency_wait();   // the kept list comes from the kernel before this one
+  grid_dependency_wait();   // the kept list (and the packed rows and norms) come from the kernel before this one
   // Nothing in global memory is written before the wait above: the kernel before this one may belong to an
   // earlier call on the same workspace and still be running.  The clear is still long before any wait can expire.
   if (m.clear_status && b == 0 && t0 == 0 && threadIdx.x == 0) *m.status = 0u;
@@ -187,7 +171,7 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
       // |m_s|^2 of the kept rows of this n-chunk, accumulated from the B stages as they pass through
       // shared memory (thread ptid owns rows ptid and ptid + 128)
       float ss[2] = {0.f, 0.f};
-      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+      for (int kc = 0; kc < (p.norms_given ? 0 : p.k_chunks); ++kc, ++it) {
         const int s = it % p.stages, round = it / p.stages;
         if (ok) ok = mbar_wait_warp(&sh.full[s], round & 1, abort_flag);
         if (!ok) continue;
@@ -212,7 +196,12 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
 #pragma unroll
       for (int u = 0; u < 2; ++u) {
         const int r = ptid + 128 * u;
-        if (r < p.n_pad) inv_norm[acc * p.n_pad + r] = (n0 + r < m.n_kept) ? 1.f / fmaxf(sqrtf(ss[u]), 1e-12f) : 0.f;
+        if (r < p.n_pad) {
+          float inv = 0.f;
+          if (n0 + r < m.n_kept)
+            inv = p.norms_given ? __ldcg(m.inv_norm + static_cast<size_t>(b) * m.n_kept + n0 + r) : 1.f / fmaxf(sqrtf(ss[u]), 1e-12f);
+          inv_norm[acc * p.n_pad + r] = inv;
+        }
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
@@ -315,7 +304,8 @@ struct PersistShared {
 
 __device__ __forceinline__ void mean_group_sync() { asm volatile("bar.sync 2, %0;" ::"n"(kMeanThreads) : "memory"); }
 
-// Packs the kept rows like pack_kept_kernel and, having read them anyway, writes 1 / max(|m_s|, eps) of every
+// Copies the kept rows of every instance into a contiguous [instance][slot][dim] buffer (slots past n_kept are
+// zero) and, having read them anyway, writes 1 / max(|m_s|, eps) of every
 // kept token; the first CTA also zeroes the status word and the counters of the persistent kernel that
 // follows.  One warp per slot, the whole row in flight at once.
 __global__ void __launch_bounds__(256) pack_kept_norm_kernel(MergeParams m, int rows_packed) {
@@ -580,6 +570,11 @@ static bool plan(const MergeParams& m, Params& p) {
   p.k_chunks = (m.metric_dim + kChunkK - 1) / kChunkK;
   p.tmem_cols = 32;   // one accumulator, or two (ping-pong) when the kept set needs several rounds
   while (p.tmem_cols < p.n_pad * (p.n_chunks > 1 ? 2 : 1)) p.tmem_cols *= 2;
+  // Large kept sets: the packing kernel has read every kept row anyway and leaves 1 / |m_s| behind; reading the
+  // B stages a second time for the norms competes with the MMAs for shared-memory bandwidth (498 us against 619 us
+  // at 2048 kept tokens).  (Two token tiles per CTA sharing every kept-row stage measured slower: 153 us against
+  // 124 us per 128 tokens, the MMAs of a round then wait for the read-back of the one before.)
+  p.norms_given = p.b_packed;
   p.a_stage_bytes = kTileM * kChunkK * 2;
   p.b_stage_bytes = ((p.n_pad * kChunkK * 2) + 1023) / 1024 * 1024;
   const int stage = p.a_stage_bytes + p.b_stage_bytes;
@@ -653,7 +648,8 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   if (st != VSCAN_OK) return st;
   if (p.b_packed) {
     dim3 pgrid((static_cast<unsigned>(p.n_chunks) * p.n_pad + 7) / 8, m.instances);
-    VSCAN_LAUNCH("pack_kept", stream, tc::pack_kept_kernel<<<pgrid, 256, 0, stream>>>(m, p.n_chunks * p.n_pad));
+    VSCAN_LAUNCH("pack_kept", stream,
+                 (void)launch_dependent(tc::pack_kept_norm_kernel, pgrid, dim3(256), 0, stream, m, p.n_chunks * p.n_pad));
   }
   const size_t smem = tc::smem_bytes(p);
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
