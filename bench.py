@@ -31,7 +31,7 @@ from synth import CONFIGS, schedule_points, stage1_inputs, stage2_inputs, sweep_
 METRIC = "VScan reduction images/s (Stage1+Stage2) at 2880 visual tokens"
 UNIT = "images/s"
 FALLBACK_HBM_GBS = 6650.0
-MERGE_KERNELS = ("kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", "merge_persistent", "pack_kept")
+MERGE_KERNELS = ("merge_cluster", "order_members", "kept_inv_norm", "assign_simt", "assign_tensor", "group_mean", "merge_persistent", "pack_kept")
 
 
 # ------------------------------------------------------------------ algorithmic work per step
@@ -386,7 +386,7 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
             "kernels": kernels,
             "merge": {"flops_per_step": merge_flops(cfg),
                       "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names),
-                      "assign_kernel": next((n for n in ("merge_persistent", "assign_tensor", "assign_simt") if n in kernels), None)},
+                      "assign_kernel": next((n for n in ("merge_cluster", "merge_persistent", "assign_tensor", "assign_simt") if n in kernels), None)},
             "gpu_launches": launches_per_step * args.steps,
             "status": status,
             "clocks": clocks,

@@ -62,6 +62,9 @@ typedef enum {
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
   VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group sums in a second
                              kernel, on the tensor cores too (one-hot matrix products) where the shape allows */
+  VSCAN_MERGE_CLUSTER = 3, /* assignment and group sums in ONE pass over the features: a cluster of dim / 256 CTAs per
+                             instance, each owning 256 feature columns, exchanges partial dot products through
+                             distributed shared memory (bf16, n_kept <= 64, dim 256 / 512 / 1024, no metric) */
   VSCAN_MERGE_INTERLEAVED = 4 /* the TENSOR path's two steps in one persistent launch, one CTA per SM: six warps
                              assign tile after tile (kept rows packed and their norms taken by a small
                              kernel first), eight more warps sum the groups of every instance whose tiles are

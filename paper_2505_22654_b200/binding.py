@@ -17,7 +17,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = ran
 F32, BF16 = 0, 1
 SCORE_ROW, SCORE_QK, SCORE_RECEIVED = 0, 1, 2
 SPAN_ONLY, SPAN_FULL = 0, 1
-MERGE_AUTO, MERGE_SIMT, MERGE_TENSOR, MERGE_INTERLEAVED = 0, 1, 2, 4
+MERGE_AUTO, MERGE_SIMT, MERGE_TENSOR, MERGE_CLUSTER, MERGE_INTERLEAVED = 0, 1, 2, 3, 4
 
 _vp, _i32, _f32 = C.c_void_p, C.c_int32, C.c_float
 

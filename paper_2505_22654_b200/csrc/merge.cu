@@ -385,7 +385,7 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
   if (!d || !d->x || !d->kept_idx || !d->merged) return VSCAN_ERR_INVALID_ARG;
   if (d->dtype != VSCAN_F32 && d->dtype != VSCAN_BF16) return VSCAN_ERR_INVALID_ARG;
   if (d->path != VSCAN_MERGE_AUTO && d->path != VSCAN_MERGE_SIMT && d->path != VSCAN_MERGE_TENSOR &&
-      d->path != VSCAN_MERGE_INTERLEAVED)
+      d->path != VSCAN_MERGE_INTERLEAVED && d->path != VSCAN_MERGE_CLUSTER)
     return VSCAN_ERR_INVALID_ARG;
   if (d->instances < 0 || d->n_tokens <= 0 || d->cls_offset < 0 || d->row_len < d->cls_offset + d->n_tokens ||
       d->dim <= 0 || d->dim % 8 || d->n_kept < 1 || d->n_kept > d->n_tokens)
@@ -471,6 +471,12 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;
   p.clear_status = 1;
+
+  // one pass over the features, a cluster per instance: on request only (see the measurements in the design notes)
+  if (d->path == VSCAN_MERGE_CLUSTER) {
+    if (!merge_cluster_supported(d->dtype, p)) return VSCAN_ERR_UNSUPPORTED;
+    return launch_merge_cluster(p, stream);
+  }
 
   // assignment and group means in one persistent launch: on request, or by itself where it measured faster
   // than the two kernels below (kept sets above 128, where those run one or two CTAs per SM)

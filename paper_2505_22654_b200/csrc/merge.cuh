@@ -39,4 +39,9 @@ bool merge_interleaved_supported(int dtype, const MergeParams& p);
 vscan_status launch_group_sum_tensor(const MergeParams& p, cudaStream_t stream);
 bool group_sum_tensor_supported(int dtype, const MergeParams& p);
 
+// Assignment and group sums in one pass over the features: a cluster of dim / 256 CTAs per instance exchanges partial
+// dot products through distributed shared memory (bf16, at most 64 kept tokens, dim 256 / 512 / 1024, no separate metric).
+vscan_status launch_merge_cluster(const MergeParams& p, cudaStream_t stream);
+bool merge_cluster_supported(int dtype, const MergeParams& p);
+
 }  // namespace vscan

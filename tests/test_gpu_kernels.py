@@ -192,6 +192,30 @@ def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
         check_merged(merged[b], m, "bf16")
 
 
+@pytest.mark.parametrize("B,N,D,K1,c", [(2, 576, 1024, 64, 1), (3, 300, 512, 17, 0), (2, 130, 256, 40, 1), (1, 1000, 1024, 33, 0),
+                                        (170, 576, 1024, 64, 1), (90, 200, 512, 9, 1)])
+def test_merge_one_pass_cluster_path(B, N, D, K1, c):
+    """The one-pass merge (a cluster of D / 256 CTAs per instance exchanging partial dot products through distributed
+    shared memory): cluster sizes 1, 2 and 4, ragged last tiles, kept counts that are not multiples of 16, and more
+    instances than clusters fit on the GPU at once (persistent loop, buffer rotation across instances)."""
+    cfg = small_cfg("bf16", grid_h=1, grid_w=N, win_h=1, win_w=N, k_w=0, k_g=K1, D=D, C=1, B=B, cls=c)
+    rng = np.random.default_rng(B * 7 + N)
+    x = round_to_dtype(rng.standard_normal((B, N + c, D)).astype(np.float32), "bf16")
+    kept = np.stack([np.sort(rng.choice(N, K1, replace=False)) for _ in range(B)])
+    check = range(B) if B <= 3 else (0, 1, B // 2, B - 2, B - 1)
+    for b in check:
+        plant.plant_merge(cfg, x[b:b + 1], kept[b:b + 1])
+    ws = vs.Workspace(64 << 20)
+    merged, assign, counts = vs.vscan_merge(dev(x, "bf16"), c, dev(kept.astype(np.int32)), want_assign=True,
+                                            want_counts=True, workspace=ws, path=vs.MERGE_CLUSTER)
+    assert vs.vscan_check(ws) == 0
+    for b in check:
+        m, a, cn = vo.merge(x[b], c, kept[b])
+        np.testing.assert_array_equal(assign[b].cpu().numpy(), a)
+        np.testing.assert_array_equal(counts[b].cpu().numpy(), cn)
+        check_merged(merged[b], m, "bf16")
+
+
 @pytest.mark.parametrize("B,N,D,K1", [(150, 200, 64, 20), (97, 131, 128, 7), (40, 576, 1024, 64)])
 def test_merge_interleaved_many_instances(B, N, D, K1):
     """More instances than the block-order distance between an instance's assignment CTAs and its mean
