@@ -166,6 +166,7 @@ def time_oracle(cfg, budget_s: float = 12.0, max_images: int = 16):
         if el >= budget_s:
             break
     return {"value": done / el, "unit": UNIT, "cores": oracle_threads(), "kind": "oracle",
+            "threads": f"1 Python thread; numpy's BLAS pool of {oracle_threads()} threads inside the matrix products",
             "sample": f"{done} images of the {cfg.name} workload ({cfg.C} crops + 1 sequence each), "
                       f"{el:.1f} s of numpy fp64"}
 
@@ -412,10 +413,39 @@ def run_vscan(args, cfg):
         run_sweep(args, rank, world, local_rank, dist)
     else:
         line = measure(args, cfg, rank, world, local_rank, dist)
+        if world == 1 and not args.no_other_workloads and args.workload == "2":
+            line["other_workloads"] = other_workloads(args, rank, world, local_rank, dist)
         if rank == 0:
             print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
+
+
+def other_workloads(args, rank, world, local_rank, dist) -> dict:
+    """Short runs of the 576-token batch workload and the 16384-token workload beside the headline line: images/s,
+    step time, step HBM fraction and, for the tensor-bound one, the assignment kernel against the sustained bf16 peak."""
+    peak_tf = 1395.5
+    try:
+        peak_tf = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"])
+    except Exception:
+        pass
+    out = {}
+    steps, sets = args.steps, args.sets
+    for idx in (1, 3):
+        cfg = CONFIGS[idx]
+        args.steps, args.sets = 20, 2
+        line = measure(args, cfg, rank, world, local_rank, dist, with_e2e=False, with_cpu=False)
+        k = line["kernels"]
+        assign = line["merge"]["assign_kernel"]
+        out[cfg.name] = {
+            "images_per_s": round(line["value"], 1), "ms_per_step": round(line["ms_per_step"], 4),
+            "step_hbm_frac": round(line["step_hbm"]["frac"], 3), "status": line["status"],
+            "kernels_us": {n: round(v["avg_us"] * v["launches_per_step"], 1) for n, v in k.items()},
+            "assign_kernel": assign,
+            "assign_frac_of_sustained_bf16": round(merge_flops(cfg) / (k[assign]["avg_us"] * 1e-6) / 1e12 / peak_tf, 3) if assign else None,
+        }
+    args.steps, args.sets = steps, sets
+    return out
 
 
 def run_sweep(args, rank, world, local_rank, dist):
@@ -437,6 +467,10 @@ def run_sweep(args, rank, world, local_rank, dist):
     points += [(label, cfg, 0, s1) for label, cfg, s1 in schedule_points()]
     if args.sweep_filter:
         points = [p for p in points if args.sweep_filter in p[0]]
+    if rank == 0 and (not args.sweep_filter or args.sweep_filter in "fma"):
+        from paper_2505_22654_b200 import binding as vb
+        print(json.dumps({"point": "fp32 fma rate (ceiling of the CUDA-core similarity path)",
+                          "tflops": round(vb.fma_rate_tflops(), 2)}), flush=True)
     if rank == 0 and (not args.sweep_filter or args.sweep_filter in "ragged"):
         import torch
         print(json.dumps(measure_ragged(args, torch.device("cuda", local_rank))), flush=True)
@@ -559,6 +593,7 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--overlap-stages", action="store_true", help="Stage 1 and Stage 2 as two parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-workloads", action="store_true", help="skip the short runs of the other named workloads")
     ap.add_argument("--sweep", action="store_true",
                     help="all named workloads, the batch x retention sweep and the paper's pruning schedules")
     ap.add_argument("--sweep-filter", default="", help="with --sweep: only the points whose label contains this")

@@ -390,6 +390,16 @@ uint64_t vscan_kernel_launches(void);
  * ------------------------------------------------------------------------------------------- */
 vscan_status vscan_selftest_bounded_wait(void* workspace, size_t workspace_bytes, uint32_t polls, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * vscan_selftest_fma_rate: a measurement aid with no counterpart in the paper.  Launches `blocks` CTAs of 256
+ * threads that each run `iters` rounds of eight independent fp32 fused multiply-adds and stores `*flops`, the
+ * floating-point operations of the launch (2 per FMA); the caller times the launch with events on `stream`.  The
+ * rate is the ceiling that the CUDA-core similarity path of vscan_merge (VSCAN_MERGE_SIMT) is held against.
+ *   scratch  device memory of at least blocks * 256 floats (overwritten)
+ * ------------------------------------------------------------------------------------------- */
+vscan_status vscan_selftest_fma_rate(float* scratch, size_t scratch_floats, int32_t blocks, int32_t iters, double* flops,
+                                     void* stream);
+
 #ifdef __cplusplus
 }
 #endif

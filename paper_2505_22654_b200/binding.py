@@ -125,6 +125,8 @@ def lib() -> C.CDLL:
         L.vscan_profile_end.argtypes = [C.c_char_p, C.POINTER(C.c_float), _i32]
         L.vscan_selftest_bounded_wait.restype = _i32
         L.vscan_selftest_bounded_wait.argtypes = [_vp, C.c_size_t, C.c_uint32, _vp]
+        L.vscan_selftest_fma_rate.restype = _i32
+        L.vscan_selftest_fma_rate.argtypes = [_vp, C.c_size_t, _i32, _i32, C.POINTER(C.c_double), _vp]
         L.vscan_score_qk_static_capacity.restype = C.c_size_t
         L.vscan_score_qk_static.restype = _i32
         L.vscan_score_qk_static.argtypes = [C.POINTER(ScoreDesc), _vp]
@@ -469,6 +471,23 @@ def profile_end(capacity: int = 4096):
         raise VScanError(ERR_INVALID_ARG, "vscan_profile_end")
     raw = names.raw
     return [(raw[i * 32:(i + 1) * 32].split(b"\0", 1)[0].decode(), float(ms[i])) for i in range(n)]
+
+
+def fma_rate_tflops(blocks: int = 148 * 16, iters: int = 1 << 15, repeats: int = 5) -> float:
+    """Measured fp32 FMA rate of the GPU in TFLOP/s (best of `repeats` launches of vscan_selftest_fma_rate)."""
+    scratch = torch.empty(blocks * 256, dtype=torch.float32, device="cuda")
+    flops = C.c_double(0.0)
+    best = 0.0
+    for _ in range(repeats + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        st = lib().vscan_selftest_fma_rate(scratch.data_ptr(), scratch.numel(), blocks, iters, C.byref(flops), _stream())
+        e1.record()
+        if st != OK:
+            raise VScanError(st, "vscan_selftest_fma_rate")
+        e1.synchronize()
+        best = max(best, flops.value / (e0.elapsed_time(e1) * 1e-3) / 1e12)
+    return best
 
 
 def vscan_check(workspace: Workspace) -> int:

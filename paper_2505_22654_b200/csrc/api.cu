@@ -33,7 +33,34 @@ void prof_after(cudaStream_t stream) {
 }
 }  // namespace vscan
 
+namespace vscan {
+// Eight independent chains of dependent fused multiply-adds per thread: what the fp32 pipes sustain, measured.
+__global__ void __launch_bounds__(256) fma_rate_kernel(float* out, int iters) {
+  float a[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) a[k] = static_cast<float>(threadIdx.x + k) * 1e-3f;
+  const float b = 1.0000001f, c = 1e-7f;
+  for (int i = 0; i < iters; ++i) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) a[k] = fmaf(a[k], b, c);
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) sum += a[k];
+  out[blockIdx.x * blockDim.x + threadIdx.x] = sum;
+}
+}  // namespace vscan
+
 using namespace vscan;
+
+extern "C" vscan_status vscan_selftest_fma_rate(float* scratch, size_t scratch_floats, int32_t blocks, int32_t iters,
+                                                double* flops, void* stream) {
+  if (!scratch || !flops || blocks <= 0 || iters <= 0 || scratch_floats < static_cast<size_t>(blocks) * 256) return VSCAN_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  VSCAN_LAUNCH("fma_rate", st, (fma_rate_kernel<<<blocks, 256, 0, st>>>(scratch, iters)));
+  *flops = 2.0 * 8.0 * 256.0 * static_cast<double>(blocks) * static_cast<double>(iters);
+  return VSCAN_OK;
+}
 
 extern "C" int32_t vscan_version(void) { return VSCAN_VERSION; }
 

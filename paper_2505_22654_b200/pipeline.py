@@ -97,7 +97,8 @@ class VScanReducer:
         """Synchronises the current stream and reads the device status words of both workspaces: 0, or
         the status a bounded device-side wait left there (binding.ERR_TIMEOUT).  A pass that timed out has
         unwritten output rows, so callers that time or trust a pass call this after it."""
-        return max(vb.vscan_check(self.ws_merge), vb.vscan_check(self.ws_prune))
+        used = [self.ws_prune] + ([self.ws_merge] if self.run_stage1 else [])   # an unused workspace holds no status
+        return max(vb.vscan_check(w) for w in used)
 
     def _reserve(self):
         import ctypes as C
