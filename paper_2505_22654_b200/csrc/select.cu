@@ -20,6 +20,8 @@ struct SelectParams {
   int n, frames, grid_h, grid_w, win_h, win_w, k_w, k_g, windows, wins_per_row, wins_per_frame;
   // ceil(2^32 / d) for d = tokens per frame, grid_w, win_h, win_w: umulhi(x, rcp) == x / d for x * d < 2^32
   uint32_t rcp_frame, rcp_grid_w, rcp_win_h, rcp_win_w;
+  // cluster form: window-row bands (win_h grid rows of one frame) handled by each CTA of a cluster
+  int bands_per_cta;
 };
 
 // Head mean of one token's attention entries, heads ascending (same arithmetic as the ROW-mode score).
@@ -327,6 +329,207 @@ __global__ void __launch_bounds__(1024) select_small_kernel(SelectParams p, int 
   if (p.kept_mask && live) p.kept_mask[static_cast<size_t>(b) * p.n + i] = keep ? 1 : 0;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Long instances: a thread-block cluster per instance.  The instance is cut into contiguous runs of whole
+// window-row bands (win_h grid rows of a frame: every window lies inside one band), one run per CTA.
+//   scores, local scan   on the CTA's own tokens only, as in select_kernel
+//   global scan          radix select over the cluster: every CTA histograms its own candidates, a cluster barrier,
+//                        then every CTA adds up the histograms of all CTAs through distributed shared memory and
+//                        takes the same decision; one histogram per pass, so one cluster barrier per pass
+//   union                every CTA publishes (tokens surely kept, candidates equal to the threshold); the counts
+//                        of the CTAs before it give the rank of its first equal key and its first output position
+// All CTAs of a cluster run the same number of cluster barriers whatever their token count; the last one keeps
+// every CTA's shared memory alive until the neighbours' remote reads are done.
+// dynamic shared memory: keys_g[cap] | keys_l[cap] | taken[cap] (bytes), cap = tokens per CTA
+struct ClusterScratch {
+  int hist[4][256];
+  int sum[4][256];      // the cluster's histogram of each pass, added up locally
+  int totals[2];        // tokens of this CTA kept for sure; its candidates equal to the threshold
+  int all_totals[8][2];
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ uint32_t cluster_nctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of the same shared-memory variable in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t peer_smem(const void* local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(local))), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ int4 ld_peer4(uint32_t addr) {
+  int4 v;
+  asm volatile("ld.shared::cluster.v4.s32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ int2 ld_peer2(uint32_t addr) {
+  int2 v;
+  asm volatile("ld.shared::cluster.v2.s32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+  return v;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(1024) select_cluster_kernel(SelectParams p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int band_tokens = p.win_h * p.grid_w;
+  const int cap = p.bands_per_cta * band_tokens;
+  uint32_t* keys_g = reinterpret_cast<uint32_t*>(smem_raw);
+  uint32_t* keys_l = keys_g + cap;
+  uint8_t* taken = reinterpret_cast<uint8_t*>(keys_l + cap);
+  __shared__ SelectScratch sc;
+  __shared__ __align__(16) ClusterScratch cs;
+  grid_dependency_launch();
+
+  const uint32_t csize = cluster_nctarank(), rank = cluster_ctarank();
+  const int b = blockIdx.x / csize;
+  const int t_lo = min(p.n, static_cast<int>(rank) * cap), t_hi = min(p.n, t_lo + cap), cnt = t_hi - t_lo;
+
+  for (int i = threadIdx.x; i < 8 * 256; i += blockDim.x) (&cs.hist[0][0])[i] = 0;   // hist and sum
+  if constexpr (std::is_void<T>::value) {
+    const float* sg = p.scores_global + static_cast<size_t>(b) * p.n + t_lo;
+    const float* sl = p.scores_local + static_cast<size_t>(b) * p.n + t_lo;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+      keys_g[i] = float_to_key(sg[i]);
+      keys_l[i] = float_to_key(sl[i]);
+      taken[i] = 0;
+    }
+  } else {
+    const size_t inst = static_cast<size_t>(b) * p.heads * p.row_len + p.cls_offset + t_lo;
+    const T* ag = static_cast<const T*>(p.attn_global) + inst;
+    const T* al = static_cast<const T*>(p.attn_local) + inst;
+    const bool same = p.attn_local == p.attn_global;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+      float g, l;
+      if (!same && p.heads == 16) {   // the common head count: all 32 loads of the token in flight at once
+        T a[16], c[16];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { a[u] = ag[i + static_cast<size_t>(u) * p.row_len]; c[u] = al[i + static_cast<size_t>(u) * p.row_len]; }
+        g = 0.f; l = 0.f;
+#pragma unroll
+        for (int u = 0; u < 16; ++u) { g += to_float(a[u]); l += to_float(c[u]); }
+        g /= 16.f; l /= 16.f;
+      } else {
+        g = head_mean_of(ag + i, p.heads, p.row_len);
+        l = same ? g : head_mean_of(al + i, p.heads, p.row_len);
+      }
+      if (p.scores_global_out) p.scores_global_out[static_cast<size_t>(b) * p.n + t_lo + i] = g;
+      if (p.scores_local_out) p.scores_local_out[static_cast<size_t>(b) * p.n + t_lo + i] = l;
+      keys_g[i] = float_to_key(g);
+      keys_l[i] = float_to_key(l);
+      taken[i] = 0;
+    }
+  }
+  __syncthreads();
+
+  // ---- local scan over the windows of this CTA's bands: one warp per window
+  if (p.k_w > 0 && cnt > 0) {
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const int m = p.win_h * p.win_w;
+    const int my_windows = (cnt / band_tokens) * p.wins_per_row;
+    for (int w = warp; w < my_windows; w += nwarps) {
+      const int band = w / p.wins_per_row, wc = w - band * p.wins_per_row;
+      const int base = band * band_tokens + wc * p.win_w;      // relative to t_lo
+      const int win_w = p.win_w, grid_w = p.grid_w;
+      auto token_of = [=](int q) { return base + (q / win_w) * grid_w + (q % win_w); };
+      if (m <= 64) warp_rank_mark(keys_l, m, p.k_w, token_of, taken);
+      else warp_select_mark(keys_l, m, p.k_w, token_of, taken);
+    }
+  }
+  __syncthreads();
+
+  // ---- global scan over the cluster's candidates
+  uint32_t thr = 0;
+  int need = 0;
+  if (p.k_g > 0) {
+    uint32_t prefix = 0, mask = 0;
+    int k_rem = p.k_g;
+    int pass = 0;
+    for (int shift = 24; shift >= 0; shift -= 8, ++pass) {
+      radix_hist_add(keys_g, taken, cnt, shift, prefix, mask, cs.hist[pass]);
+      cluster_barrier();                     // every CTA's histogram of this pass is complete and visible
+      {   // warp c fetches the histogram of CTA c (all remote reads in flight together) and adds it to the local sum
+        const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        if (warp < csize) {
+          const uint32_t addr = peer_smem(&cs.hist[pass][lane * 8], warp);
+          const int4 lo4 = ld_peer4(addr), hi4 = ld_peer4(addr + 16);
+          int* dst = &cs.sum[pass][lane * 8];
+          atomicAdd(dst + 0, lo4.x); atomicAdd(dst + 1, lo4.y); atomicAdd(dst + 2, lo4.z); atomicAdd(dst + 3, lo4.w);
+          atomicAdd(dst + 4, hi4.x); atomicAdd(dst + 5, hi4.y); atomicAdd(dst + 6, hi4.z); atomicAdd(dst + 7, hi4.w);
+        }
+      }
+      __syncthreads();
+      if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        int local[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) local[j] = cs.sum[pass][lane * 8 + j];
+        radix_pick(local, lane, k_rem, prefix, shift, sc);
+      }
+      __syncthreads();
+      prefix = sc.threshold;
+      k_rem = sc.need;
+      mask |= 0xFFu << shift;
+      __syncthreads();
+    }
+    thr = prefix;
+    need = k_rem;
+  }
+
+  // ---- union, ascending.  Each thread owns a contiguous run of this CTA's tokens.
+  const int per = (cnt + blockDim.x - 1) / blockDim.x;
+  const int lo = min(cnt, static_cast<int>(threadIdx.x) * per), hi = min(cnt, lo + per);
+  int sure_local = 0, eq_local = 0;
+  for (int i = lo; i < hi; ++i) {
+    const bool cand = !taken[i] && p.k_g > 0;
+    sure_local += taken[i] || (cand && keys_g[i] > thr);
+    eq_local += cand && keys_g[i] == thr;
+  }
+  int sure_total, eq_total;
+  int sure_before = block_exclusive_scan(sure_local, sc.warp_sums, sure_total);
+  int eq_before = block_exclusive_scan(eq_local, sc.warp_sums, eq_total);
+  if (threadIdx.x == 0) { cs.totals[0] = sure_total; cs.totals[1] = eq_total; }
+  cluster_barrier();
+  if (threadIdx.x < csize) {
+    const int2 t = ld_peer2(peer_smem(&cs.totals[0], threadIdx.x));
+    cs.all_totals[threadIdx.x][0] = t.x; cs.all_totals[threadIdx.x][1] = t.y;
+  }
+  __syncthreads();
+  int eq_base = 0, pos_base = 0;
+  for (uint32_t c = 0; c < rank; ++c) {
+    const int e = cs.all_totals[c][1];
+    pos_base += cs.all_totals[c][0] + min(max(need - eq_base, 0), e);
+    eq_base += e;
+  }
+  eq_before += eq_base;
+  // position of this thread's first kept token: the sure ones before it plus the equal keys before it that made it
+  int pos = pos_base + sure_before + (min(eq_before, need) - min(eq_base, need));
+  const int k1 = p.windows * p.k_w + p.k_g;
+  int32_t* out = p.kept_idx + static_cast<size_t>(b) * k1;
+  uint8_t* mk = p.kept_mask ? p.kept_mask + static_cast<size_t>(b) * p.n + t_lo : nullptr;
+  for (int i = lo; i < hi; ++i) {
+    bool keep = taken[i];
+    if (!keep && p.k_g > 0) {
+      const uint32_t key = keys_g[i];
+      if (key > thr) keep = true;
+      else if (key == thr) { keep = eq_before < need; ++eq_before; }
+    }
+    if (keep) { if (pos < k1) out[pos] = t_lo + i; ++pos; }
+    if (mk) mk[i] = keep ? 1 : 0;
+  }
+  cluster_barrier();   // nobody leaves while a neighbour may still read its histograms or counts
+}
+
 }  // namespace vscan
 
 using namespace vscan;
@@ -386,6 +589,47 @@ static size_t stage_block_bytes(const vscan_score_select_desc* d, long long n) {
   return bytes;
 }
 
+// ---- the cluster kernel: instances above kClusterSelect tokens that have at least two window-row bands
+constexpr long long kClusterSelect = 2048;
+constexpr int kMaxSelectCluster = 8;      // the portable cluster size (16, non-portable, measured no faster)
+// CTAs per instance: enough that a CTA holds about a thousand tokens, at most one per band.  0 = not applicable.
+static int select_cluster_size(const vscan_select_desc* d, long long n, int max_size, int* bands_per_cta) {
+  if (n <= kClusterSelect) return 0;
+  const int bands = d->frames * (d->grid_h / d->win_h);
+  if (bands < 2) return 0;
+  int c = static_cast<int>((n + 1023) / 1024);
+  if (c > max_size) c = max_size;
+  if (c > bands) c = bands;
+  const int per = (bands + c - 1) / c;
+  c = (bands + per - 1) / per;             // no CTA without a band
+  *bands_per_cta = per;
+  return c >= 2 ? c : 0;
+}
+
+template <typename T>
+static vscan_status launch_select_cluster(const char* name, SelectParams& p, const vscan_select_desc* d, cudaStream_t st) {
+  const int instances = d->instances;
+  const int csize = select_cluster_size(d, p.n, kMaxSelectCluster, &p.bands_per_cta);
+  const size_t cap = static_cast<size_t>(p.bands_per_cta) * p.win_h * p.grid_w;
+  const size_t smem = cap * 9 + 16;
+  if (smem > kMaxDynamicSmem) return VSCAN_ERR_UNSUPPORTED;
+  VSCAN_CUDA_TRY(allow_smem(select_cluster_kernel<T>, smem));
+  cudaLaunchConfig_t cfg = {};
+  int threads = static_cast<int>((cap + 31) / 32 * 32);
+  threads = threads > 1024 ? 1024 : (threads < 256 ? 256 : threads);
+  cfg.gridDim = dim3(static_cast<unsigned>(instances) * csize);
+  cfg.blockDim = dim3(threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  VSCAN_LAUNCH(name, st, (void)cudaLaunchKernelEx(&cfg, select_cluster_kernel<T>, p));
+  return VSCAN_OK;
+}
+
 extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, void* /*workspace*/,
                                                   size_t /*workspace_bytes*/, void* stream) {
   if (d && d->instances == 0) return VSCAN_OK;  // empty batch
@@ -410,6 +654,8 @@ extern "C" vscan_status vscan_select_global_local(const vscan_select_desc* d, vo
     VSCAN_LAUNCH("select", st, select_small_kernel<void><<<d->instances, small_threads(n), small_smem(n, 0, false), st>>>(p, 0));
     return VSCAN_OK;
   }
+  int unused;
+  if (select_cluster_size(d, n, kMaxSelectCluster, &unused)) return launch_select_cluster<void>("select", p, d, st);
   const size_t smem = static_cast<size_t>(n) * 9 + 16;
   VSCAN_CUDA_TRY(allow_smem(select_kernel<void>, smem));
   VSCAN_LAUNCH("select", st, select_kernel<void><<<d->instances, select_threads(n, windows), smem, st>>>(p));
@@ -461,6 +707,11 @@ extern "C" vscan_status vscan_score_select(const vscan_score_select_desc* d, voi
       VSCAN_LAUNCH("score_select", st, select_small_kernel<__nv_bfloat16><<<sd->instances, small_threads(n), sm, st>>>(p, static_cast<int>(stage)));
     }
     return VSCAN_OK;
+  }
+  int unused;
+  if (select_cluster_size(sd, n, kMaxSelectCluster, &unused)) {
+    if (d->dtype == VSCAN_F32) return launch_select_cluster<float>("score_select", p, sd, st);
+    return launch_select_cluster<__nv_bfloat16>("score_select", p, sd, st);
   }
   const size_t smem = static_cast<size_t>(n) * 9 + 16;
   const int threads = select_threads(n, windows);

@@ -17,6 +17,69 @@ struct SelectScratch {
   int need;
 };
 
+// One pass of the radix select, first half: every candidate whose bits above the current digit equal
+// `prefix` adds one to hist[digit].  hist must be zero; the caller synchronises before reading it.
+__device__ __forceinline__ void radix_hist_add(const uint32_t* keys, const uint8_t* excluded, int n, int shift,
+                                               uint32_t prefix, uint32_t mask, int* hist) {
+  // Scores of one instance share their exponent, so in the first pass nearly every key falls into
+  // the same bin: there lanes with equal digits are counted with one shared-memory atomic per warp.
+  // Later passes see spread-out digits and add directly.
+  if (shift == 24) {
+    for (int base = 0; base < n; base += blockDim.x) {
+      const int i = base + threadIdx.x;
+      const bool valid = i < n && !(excluded && excluded[i]);
+      const uint32_t digit = valid ? (keys[i] >> 24) : 0u;
+      // the lanes that share the digit of the warp's first candidate are counted with one atomic, the
+      // others (few) add one by one
+      const unsigned lane = threadIdx.x & 31;
+      const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+      if (vmask) {
+        const int lead = __ffs(vmask) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, lead);
+        const unsigned same = __ballot_sync(0xffffffffu, valid && digit == d0);
+        if (lane == static_cast<unsigned>(lead)) atomicAdd(&hist[d0], __popc(same));
+        if (valid && digit != d0) atomicAdd(&hist[digit], 1);
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+      if (excluded && excluded[i]) continue;
+      const uint32_t key = keys[i];
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+    }
+  }
+}
+
+// Second half, one warp: lane l holds the counts of bins [8l, 8l+8) in local[]; the bin that holds the
+// k_rem-th largest candidate extends the prefix, and the candidates above it inside the bin are taken off
+// k_rem.  The owning lane writes sc.threshold / sc.need.
+__device__ __forceinline__ void radix_pick(const int (&local)[8], int lane, int k_rem, uint32_t prefix, int shift,
+                                           SelectScratch& sc) {
+  int sum = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) sum += local[j];
+  // above = candidates in bins owned by higher lanes
+  int incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    int t = __shfl_down_sync(0xffffffffu, incl, o);
+    if (lane + o < 32) incl += t;
+  }
+  int above = incl - sum;
+  // the k_rem-th largest lies in this lane's bins iff above < k_rem <= above + sum
+  if (above < k_rem && k_rem <= above + sum) {
+    int acc = above;
+#pragma unroll
+    for (int j = 7; j >= 0; --j) {
+      if (acc < k_rem && k_rem <= acc + local[j]) {
+        sc.threshold = prefix | (static_cast<uint32_t>(lane * 8 + j) << shift);
+        sc.need = k_rem - acc;
+      }
+      acc += local[j];
+    }
+  }
+}
+
 // Block-wide radix select, 4 passes of 8 bits.  Candidates are the i in [0, n) with
 // excluded == nullptr || !excluded[i].  Requires 1 <= k <= #candidates.  All threads of the
 // block must call; on return every thread reads the same (threshold, need).
@@ -28,60 +91,15 @@ __device__ __forceinline__ void block_radix_select(const uint32_t* keys, const u
   for (int shift = 24; shift >= 0; shift -= 8) {
     for (int i = threadIdx.x; i < 256; i += blockDim.x) sc.hist[i] = 0;
     __syncthreads();
-    // Scores of one instance share their exponent, so in the first pass nearly every key falls into
-    // the same bin: there lanes with equal digits are counted with one shared-memory atomic per warp.
-    // Later passes see spread-out digits and add directly.
-    if (shift == 24) {
-      for (int base = 0; base < n; base += blockDim.x) {
-        const int i = base + threadIdx.x;
-        const bool valid = i < n && !(excluded && excluded[i]);
-        const uint32_t digit = valid ? (keys[i] >> 24) : 0u;
-        // the lanes that share the digit of the warp's first candidate are counted with one atomic, the
-        // others (few) add one by one
-        const unsigned lane = threadIdx.x & 31;
-        const unsigned vmask = __ballot_sync(0xffffffffu, valid);
-        if (vmask) {
-          const int lead = __ffs(vmask) - 1;
-          const uint32_t d0 = __shfl_sync(0xffffffffu, digit, lead);
-          const unsigned same = __ballot_sync(0xffffffffu, valid && digit == d0);
-          if (lane == static_cast<unsigned>(lead)) atomicAdd(&sc.hist[d0], __popc(same));
-          if (valid && digit != d0) atomicAdd(&sc.hist[digit], 1);
-        }
-      }
-    } else {
-      for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        if (excluded && excluded[i]) continue;
-        const uint32_t key = keys[i];
-        if ((key & mask) == prefix) atomicAdd(&sc.hist[(key >> shift) & 255u], 1);
-      }
-    }
+    radix_hist_add(keys, excluded, n, shift, prefix, mask, sc.hist);
     __syncthreads();
     if (threadIdx.x < 32) {
       // lane l owns bins [8l, 8l+8); walk from the top bin down
       const int lane = threadIdx.x;
-      int local[8], sum = 0;
+      int local[8];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { local[j] = sc.hist[lane * 8 + j]; sum += local[j]; }
-      // above = candidates in bins owned by higher lanes
-      int incl = sum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        int t = __shfl_down_sync(0xffffffffu, incl, o);
-        if (lane + o < 32) incl += t;
-      }
-      int above = incl - sum;
-      // the k_rem-th largest lies in this lane's bins iff above < k_rem <= above + sum
-      if (above < k_rem && k_rem <= above + sum) {
-        int acc = above;
-#pragma unroll
-        for (int j = 7; j >= 0; --j) {
-          if (acc < k_rem && k_rem <= acc + local[j]) {
-            sc.threshold = prefix | (static_cast<uint32_t>(lane * 8 + j) << shift);
-            sc.need = k_rem - acc;
-          }
-          acc += local[j];
-        }
-      }
+      for (int j = 0; j < 8; ++j) local[j] = sc.hist[lane * 8 + j];
+      radix_pick(local, lane, k_rem, prefix, shift, sc);
     }
     __syncthreads();
     prefix = sc.threshold;

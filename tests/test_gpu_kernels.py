@@ -46,6 +46,10 @@ SELECT_SHAPES = [  # F, Gh, Gw, wh, ww, k_w, k_g
     (1, 24, 24, 6, 6, 2, 32), (1, 24, 24, 6, 6, 6, 96), (1, 24, 24, 6, 6, 0, 64), (1, 24, 24, 6, 6, 3, 0),
     (1, 24, 24, 24, 24, 10, 5), (2, 4, 6, 2, 3, 1, 3), (1, 1, 1, 1, 1, 1, 0), (1, 5, 7, 1, 1, 0, 35),
     (3, 10, 10, 5, 2, 4, 100), (16, 32, 32, 8, 8, 4, 1024), (1, 24, 24, 6, 6, 36, 0), (4, 16, 16, 16, 16, 37, 11),
+    # above 2048 tokens a cluster of CTAs shares an instance: uneven band counts per CTA, windows above 64 tokens,
+    # no local or no global scan, a global scan that takes everything left
+    (5, 24, 24, 6, 6, 2, 300), (3, 30, 30, 10, 30, 0, 500), (1, 64, 48, 2, 48, 50, 0), (7, 20, 20, 4, 5, 1, 2000),
+    (16, 32, 32, 32, 32, 9, 16240), (1, 128, 128, 64, 128, 3, 77),
 ]
 
 
@@ -81,7 +85,8 @@ def test_select_uniform_scores_take_first_indices_and_aliasing():
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("shape", [(1, 24, 24, 6, 6, 2, 32, 1, 16), (2, 6, 8, 3, 4, 5, 20, 0, 5),
-                                   (1, 16, 16, 16, 16, 40, 9, 1, 3), (16, 32, 32, 8, 8, 4, 1024, 0, 16)])
+                                   (1, 16, 16, 16, 16, 40, 9, 1, 3), (16, 32, 32, 8, 8, 4, 1024, 0, 16),
+                                   (5, 24, 24, 6, 6, 2, 300, 1, 16), (3, 30, 30, 10, 30, 7, 500, 0, 5)])
 def test_score_select_fused_matches_oracle(dtype, shape):
     F, Gh, Gw, wh, ww, k_w, k_g, c, H = shape
     N, B = F * Gh * Gw, 2
