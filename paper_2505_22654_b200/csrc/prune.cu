@@ -105,11 +105,12 @@ constexpr int kPruneThreads = 128;
 constexpr unsigned kReadySpinLimit = 1u << 22;
 
 template <typename T, int VPS>
-__global__ void __launch_bounds__(kPruneThreads) prune_fused_kernel(QkParams q, CompactParams c, int n_score) {
+__global__ void __launch_bounds__(kPruneThreads, 8) prune_fused_kernel(QkParams q, CompactParams c, int n_score) {
   extern __shared__ __align__(16) float smem_f[];
   const int blk = blockIdx.x;
   if (blk < n_score) {
-    qk_softmax_role<T, VPS>(q, blk % q.q_heads, blk / q.q_heads, smem_f);
+    const int unit = blk / q.nsplit;   // (sequence, head), heads fastest; the shares of a unit are neighbours
+    qk_softmax_role<T, VPS>(q, unit % q.q_heads, unit / q.q_heads, smem_f, blk - unit * q.nsplit);
     return;
   }
   int idx = blk - n_score;
@@ -143,7 +144,7 @@ __global__ void __launch_bounds__(kPruneThreads) prune_fused_kernel(QkParams q, 
 template <typename T>
 static vscan_status launch_prune_fused(const QkParams& q, const CompactParams& c, size_t smem, cudaStream_t stream) {
   constexpr int E = Vec16<T>::kElems;
-  const int n_score = c.batch * q.q_heads;
+  const int n_score = c.batch * q.q_heads * q.nsplit;
   const unsigned blocks = static_cast<unsigned>(n_score) + static_cast<unsigned>(c.batch) * c.seq_out;
   const int vecs = q.head_dim / E;
 #define VSCAN_PRUNE_CASE(VPS)                                                                                  \
@@ -219,9 +220,27 @@ static vscan_status validate_prune(const vscan_prune_desc* d) {
   return VSCAN_OK;
 }
 
+// CTAs that share the keys of one (head, sequence) in the scoring part: one per 256 keys, at most 8, and only while
+// the scoring CTAs of the whole batch stay within what the SMs hold at once (a few long sequences).
+static int score_splits(const vscan_prune_desc* d) {
+  const long long soft_n = d->softmax_span == VSCAN_SPAN_ONLY ? d->n_vis : 1ll * d->n_sys + d->n_vis + d->n_txt;
+  long long n = soft_n / 256;
+  n = n > 8 ? 8 : n;
+  const long long units = 1ll * d->batch * d->q_heads;
+  while (n > 1 && units * n > 1184) --n;   // 8 scoring CTAs per SM
+  return n < 1 ? 1 : static_cast<int>(n);
+}
+// per-sequence arrival counters and ready flags, per-(sequence, head) tickets of the split form
+static size_t prune_counter_bytes(const vscan_prune_desc* d) {
+  return round_up((2 + static_cast<size_t>(d->q_heads)) * d->batch * sizeof(int), 256);
+}
+static size_t prune_stats_bytes(const vscan_prune_desc* d) {
+  return round_up(static_cast<size_t>(d->batch) * d->q_heads * 8 * sizeof(float2), 256);
+}
+
 extern "C" size_t vscan_llm_prune_workspace_bytes(const vscan_prune_desc* d) {
   if (!d || d->batch <= 0 || d->q_heads <= 0 || d->n_vis <= 0) return kStatusBytes;
-  return kStatusBytes + round_up(2 * static_cast<size_t>(d->batch) * sizeof(int), 256) +
+  return kStatusBytes + prune_counter_bytes(d) + prune_stats_bytes(d) +
          round_up(static_cast<size_t>(d->batch) * d->q_heads * d->n_vis * sizeof(float), 256);
 }
 
@@ -235,9 +254,10 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
   const size_t need = vscan_llm_prune_workspace_bytes(d);
   if (!workspace || !aligned256(workspace) || workspace_bytes < need) return VSCAN_ERR_WORKSPACE;
   const int seq_len = d->n_sys + d->n_vis + d->n_txt, seq_out = seq_len - d->n_vis + d->k_keep;
-  // workspace: status word | per-sequence arrival counters, per-sequence ready flags | per-head probabilities
+  // workspace: status word | per-sequence arrival counters, per-sequence ready flags, per-head tickets |
+  //            (max, sum) of the key shares | per-head probabilities
   char* ws = static_cast<char*>(workspace);
-  const size_t counter_bytes = round_up(2 * static_cast<size_t>(d->batch) * sizeof(int), 256);
+  const size_t counter_bytes = prune_counter_bytes(d);
   const size_t e = dtype_bytes(d->dtype);
   CompactParams c;
   c.kept_vis = d->kept_vis;
@@ -256,7 +276,9 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
     p.q = d->q_last; p.k = d->k; p.status = static_cast<uint32_t*>(workspace);
     p.counters = reinterpret_cast<int*>(ws + kStatusBytes);
     p.ready = p.counters + d->batch;
-    p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes);
+    p.head_tickets = p.ready + d->batch;
+    p.stats = reinterpret_cast<float2*>(ws + kStatusBytes + counter_bytes);
+    p.probs = reinterpret_cast<float*>(ws + kStatusBytes + counter_bytes + prune_stats_bytes(d));
     p.scores = d->scores; p.kept = d->kept_vis; p.k_keep = d->k_keep;
     p.q_heads = d->q_heads; p.kv_heads = d->kv_heads; p.seq_len = seq_len; p.head_dim = d->head_dim;
     p.span_begin = d->n_sys; p.span_len = d->n_vis; p.scale = d->scale;
@@ -264,9 +286,11 @@ extern "C" vscan_status vscan_llm_prune(const vscan_prune_desc* d, void* workspa
     else { p.soft_lo = 0; p.soft_n = seq_len; }
     VSCAN_CUDA_TRY(cudaMemsetAsync(p.counters, 0, counter_bytes, stream));
     // one launch for score, top-k and compaction when the top-k fits the 128-thread scoring CTAs
-    const long long blocks = 1ll * d->batch * d->q_heads + 1ll * d->batch * seq_out;
+    const int nsplit = score_splits(d);
+    const long long blocks = 1ll * d->batch * d->q_heads * nsplit + 1ll * d->batch * seq_out;
     const size_t smem = qk_smem_bytes(p.head_dim, p.soft_n);
     if (d->n_vis <= 8192 && seq_out > 0 && blocks < (1ll << 31) && smem <= kMaxDynamicSmem) {
+      p.nsplit = nsplit;
       st = d->dtype == VSCAN_F32 ? launch_prune_fused<float>(p, c, smem, stream)
                                  : launch_prune_fused<__nv_bfloat16>(p, c, smem, stream);
       if (st != VSCAN_OK) return st;

@@ -406,6 +406,33 @@ def test_llm_prune_small_planted(dtype, span):
         np.testing.assert_array_equal(out["pos"][:, b].cpu().numpy(), case["pos_ids"][:, b][:, rows])
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("span", [vo.SPAN_ONLY, vo.SPAN_FULL])
+@pytest.mark.parametrize("n_sys,n_vis,n_txt", [(5, 1100, 9), (0, 2048, 0), (300, 513, 260)])
+def test_llm_prune_long_sequences_share_a_head_between_ctas(dtype, span, n_sys, n_vis, n_txt):
+    """A few long sequences: several CTAs take contiguous shares of one head's keys and the last to finish rescales
+    the row (Eq. 5 is unchanged: the softmax over the span from the shares' maxima and sums).  Shares that straddle
+    the span's ends, a span that is the whole sequence, text and system keys that only enter the denominator."""
+    B, Hq, Hkv, d, Dh, k_keep = 2, 6, 3, 64, 32, 200
+    S = n_sys + n_vis + n_txt
+    q = round_to_dtype(RNG.standard_normal((B, Hq, d)).astype(np.float32), dtype)
+    k = round_to_dtype(RNG.standard_normal((B, Hkv, S, d)).astype(np.float32), dtype)
+    h = round_to_dtype(RNG.standard_normal((B, S, Dh)).astype(np.float32), dtype)
+    pos = np.tile(np.arange(S, dtype=np.int32), (1, B, 1))
+    scale = 0.5
+    out = vs.vscan_llm_prune(dev(q, dtype), dev(k, dtype), None, dev(h, dtype), dev(pos), n_sys, n_vis, n_txt, k_keep,
+                             scale, span, want_scores=True)
+    s32 = out["scores"].cpu().numpy()
+    for b in range(B):
+        ref = vo.score_qk(q[b], k[b], n_sys, n_vis, scale, span)
+        assert np.abs(s32[b] - ref).max() <= TOL_SCORE
+        kept = out["kept_vis"][b].cpu().numpy()
+        np.testing.assert_array_equal(kept, vo.topk_lowest_index(s32[b], k_keep))   # decided on the kernel's fp32 scores
+        rows = vo.compaction_rows(n_sys, n_vis, n_txt, kept)
+        np.testing.assert_array_equal(out["hidden"][b].float().cpu().numpy(), h[b][rows])
+        np.testing.assert_array_equal(out["k"][b].float().cpu().numpy(), k[b][:, rows])
+
+
 def test_multi_turn_reselection_from_the_same_pool():
     """App. B "multi-turn conversations": a new question re-scores and re-selects from the existing
     token pool.  The library is stateless, so this is a second call with the new last-token query on
