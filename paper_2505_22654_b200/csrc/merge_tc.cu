@@ -269,6 +269,180 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
   assign_tile(&map_a, &map_b, p, sh, smem_dyn, blockIdx.y, blockIdx.x * kTileM, nullptr);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Large kept sets (packed rows, norms from the packing kernel): the assignment on CTA pairs.  A pair of CTAs
+// (a cluster of two, on the two SMs of one TPC) takes 256 tokens; each CTA loads its own 128 token rows and HALF of
+// the kept rows of a stage, and one MMA of M = 256 issued by the even CTA runs on both SMs, each tensor core reading
+// its own token tile and both halves of the kept rows.  Per 128 tokens and stage an SM takes in 16 KB + n_pad/2 rows
+// instead of 16 KB + n_pad rows, which is what bounds the single-CTA form at these sizes.
+//   warp 0 (both CTAs)   producer: waits on its own `empty`, loads into its own shared memory, bytes counted on
+//                        the leader's `full` (armed by the leader's producer with the bytes of both CTAs)
+//   warp 1 (leader)      MMA issuer; after a stage's MMAs one commit per CTA frees the stage in both, after an
+//                        n-chunk one commit per CTA publishes the accumulator in both
+//   warps 2-5 (both)     read their CTA's 128 accumulator rows, running arg-max; the release of an accumulator is
+//                        an arrive on the leader's `tmem_empty` (count 8: four warps of each CTA)
+// Tensor memory is allocated and freed by warp 1 of both CTAs (pair-wide allocation); a cluster barrier before the
+// release makes sure neither CTA leaves, or frees anything, while the other may still use it.  Every mbarrier wait
+// is bounded as in assign_tile.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads)
+assign_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p) {
+  extern __shared__ unsigned char smem_dyn[];
+  __shared__ Shared sh;
+  unsigned char* tiles = smem_dyn + ((1024u - (static_cast<uint32_t>(__cvta_generic_to_shared(smem_dyn)) & 1023u)) & 1023u);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const MergeParams& m = p.m;
+  const uint32_t rank = pair_rank();
+  const bool leader = rank == 0;
+  const int b = blockIdx.y, t0 = (blockIdx.x >> 1) * (2 * kTileM) + static_cast<int>(rank) * kTileM;
+  volatile int* abort_flag = &sh.abort_flag;
+  const int half_rows = p.n_pad / 2;                              // kept rows of a stage held by this CTA
+  const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;      // b_stage_bytes: half_rows * 128, rounded to 1024
+  float* inv_norm = reinterpret_cast<float*>(tiles + p.stages * stage_bytes);   // [accumulator][n_pad]
+  const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 8); }
+    sh.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh.tmem_base)), "r"(p.tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  pair_sync();   // both CTAs' barriers exist before either sends a load or an arrive to the other
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_acc = sh.tmem_base;
+  grid_dependency_launch();
+  grid_dependency_wait();   // kept list, packed rows and norms come from the kernels before this one; nothing is written before
+  if (m.clear_status && b == 0 && blockIdx.x == 0 && threadIdx.x == 0) *m.status = 0u;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    int it = 0;
+    bool ok = true;
+    for (int nc = 0; nc < p.n_chunks; ++nc) {
+      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+        const int s = it % p.stages, round = it / p.stages;
+        if (ok && round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
+        if (!ok) continue;
+        if (lane == 0) {
+          unsigned char* at = tiles + s * stage_bytes;
+          if (leader) mbar_arrive_expect_tx(&sh.full[s], 2u * static_cast<uint32_t>(p.a_stage_bytes + half_rows * 128));
+          const uint32_t bar = pair_addr(&sh.full[s], 0);
+          pair_tma_load_3d(at, &map_a, bar, kc * kChunkK, m.cls_offset + t0, b);
+          pair_tma_load_3d(at + p.a_stage_bytes, &map_b, bar, kc * kChunkK, nc * p.n_pad + static_cast<int>(rank) * half_rows, b);
+        }
+      }
+    }
+    // the leader's commits to this CTA's `empty` barriers have all arrived before its shared memory goes
+    for (int i = max(0, it - p.stages); i < it; ++i)
+      if (ok) ok = mbar_wait_warp(&sh.empty[i % p.stages], (i / p.stages) & 1, abort_flag);
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (leader only)
+    if (leader && lane == 0) {
+      const uint32_t idesc = pair_instr_desc_bf16(p.n_pad);
+      int it = 0;
+      for (int nc = 0; nc < p.n_chunks && !*abort_flag; ++nc) {
+        const int acc = nc & 1, use = nc >> 1;
+        if (use > 0) {
+          if (!mbar_wait(&sh.tmem_empty[acc], (use - 1) & 1, abort_flag)) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        }
+        const uint32_t d_addr = tmem_acc + acc * p.n_pad;
+        bool ok = true;
+        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+          const int s = it % p.stages, round = it / p.stages;
+          if (!mbar_wait(&sh.full[s], round & 1, abort_flag)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = smem_u32(tiles + s * stage_bytes), b_addr = a_addr + p.a_stage_bytes;
+          const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
+#pragma unroll
+          for (int k = 0; k < kChunkK / 16; ++k)
+            pair_umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
+          pair_umma_commit(smem_u32(&sh.empty[s]));
+          pair_umma_commit(pair_addr(&sh.empty[s], 1));
+        }
+        if (!ok) break;
+        pair_umma_commit(smem_u32(&sh.tmem_full[acc]));
+        pair_umma_commit(pair_addr(&sh.tmem_full[acc], 1));
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------ epilogue: this CTA's 128 accumulator rows -> arg-max
+    const int ptid = (warp - 2) * 32 + lane;
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    float best_val = -INFINITY;
+    int best_idx = 0;
+    bool ok = true;
+    for (int nc = 0; nc < p.n_chunks; ++nc) {
+      const int n0 = nc * p.n_pad, acc = nc & 1, use = nc >> 1;
+#pragma unroll
+      for (int u = 0; u < 2; ++u) {
+        const int r = ptid + 128 * u;
+        if (r < p.n_pad)
+          inv_norm[acc * p.n_pad + r] = n0 + r < m.n_kept ? __ldcg(m.inv_norm + static_cast<size_t>(b) * m.n_kept + n0 + r) : 0.f;
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
+      if (!ok) continue;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.n_pad;
+      for (int c0 = 0; c0 < p.n_pad; c0 += 32) {
+        uint32_t v[32];
+        if (p.n_pad - c0 >= 32) tmem_ld32(taddr + c0, v);
+        else {
+          tmem_ld16(taddr + c0, v);
+#pragma unroll
+          for (int j = 16; j < 32; ++j) v[j] = 0u;
+        }
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int s_idx = n0 + c0 + j;
+          if (c0 + j < p.n_pad && s_idx < m.n_kept) {
+            const float val = __uint_as_float(v[j]) * inv_norm[acc * p.n_pad + c0 + j];
+            if (val > best_val) { best_val = val; best_idx = s_idx; }
+          }
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) {
+        if (leader) mbar_arrive(&sh.tmem_empty[acc]);
+        else pair_remote_arrive(pair_addr(&sh.tmem_empty[acc], 0));
+      }
+    }
+    sh.best_slot[row] = best_idx;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    for (int s_idx = ptid; s_idx < m.n_kept; s_idx += 128) {   // a kept token belongs to its own slot
+      const int t = min(max(kept[s_idx], 0), m.n_tokens - 1);
+      if (t >= t0 && t < t0 + kTileM) sh.best_slot[t - t0] = s_idx;
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (ok && t0 + ptid < m.n_tokens) m.assign[static_cast<size_t>(b) * m.n_tokens + t0 + ptid] = sh.best_slot[ptid];
+  }
+
+  // ------------------------------------------------------------ teardown
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (sh.abort_flag) {
+    if (threadIdx.x == 0) atomicExch(m.status, static_cast<uint32_t>(VSCAN_ERR_TIMEOUT));
+    for (int i = 0; i < 64; ++i) __nanosleep(2000);   // copies still in flight land before the shared memory goes
+    __syncthreads();
+  }
+  pair_sync();   // the other CTA's MMAs, loads and tensor-memory reads are over as well
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(p.tmem_cols) : "memory");
+  }
+}
+
 // Assignment and group means in ONE persistent launch (one CTA per SM), so that the second pass over the
 // features (the sums of Eq. 4) reads them from L2 while they are still there, the start-up cost of a CTA
 // is paid once per SM instead of once per tile, and the read-back of one tile overlaps the MMAs of the next.
@@ -606,7 +780,7 @@ bool assign_tensor_supported(int dtype, const MergeParams& m) {
 
 // Tensor maps of a launch: the token tiles (3-D [instance][row][dim]) and the kept rows (the same memory
 // as a 2-D [all rows][dim] tensor for row gathers, or the packed copy for large kept sets).
-static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUtensorMap& map, CUtensorMap& map_b) {
+static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUtensorMap& map, CUtensorMap& map_b, int packed_box_rows) {
   tc::EncodeTiledFn encode = tc::encode_fn();
   if (!encode) return VSCAN_ERR_UNSUPPORTED;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(m.metric_dim), static_cast<cuuint64_t>(m.row_len),
@@ -628,7 +802,7 @@ static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUten
     const cuuint64_t rows_packed = static_cast<cuuint64_t>(p.n_chunks) * p.n_pad;
     const cuuint64_t dims_p[3] = {static_cast<cuuint64_t>(m.metric_dim), rows_packed, static_cast<cuuint64_t>(m.instances)};
     const cuuint64_t strides_p[2] = {static_cast<cuuint64_t>(m.metric_dim) * 2, rows_packed * m.metric_dim * 2};
-    const cuuint32_t box_p[3] = {tc::kChunkK, static_cast<cuuint32_t>(p.n_pad), 1};
+    const cuuint32_t box_p[3] = {tc::kChunkK, static_cast<cuuint32_t>(packed_box_rows), 1};
     r = encode(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, m.kept_packed, dims_p, strides_p, box_p, elem,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -643,13 +817,28 @@ static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUten
 vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   tc::Params p;
   if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
+  // packed kept rows: CTA pairs, each CTA holding half of a stage's kept rows
+  const bool pair = p.b_packed && p.norms_given && p.n_pad % 16 == 0;
+  if (pair) {
+    p.b_stage_bytes = ((p.n_pad / 2 * tc::kChunkK * 2) + 1023) / 1024 * 1024;
+    int stages = (215 * 1024) / (p.a_stage_bytes + p.b_stage_bytes);
+    p.stages = stages > tc::kMaxStages ? tc::kMaxStages : stages;
+  }
   CUtensorMap map, map_b;
-  vscan_status st = encode_maps(m, p, map, map_b);
+  vscan_status st = encode_maps(m, p, map, map_b, pair ? p.n_pad / 2 : p.n_pad);
   if (st != VSCAN_OK) return st;
   if (p.b_packed) {
     dim3 pgrid((static_cast<unsigned>(p.n_chunks) * p.n_pad + 7) / 8, m.instances);
     VSCAN_LAUNCH("pack_kept", stream,
                  (void)launch_dependent(tc::pack_kept_norm_kernel, pgrid, dim3(256), 0, stream, m, p.n_chunks * p.n_pad));
+  }
+  if (pair) {
+    const size_t smem = tc::smem_bytes(p);
+    VSCAN_CUDA_TRY(allow_smem(tc::assign_pair_kernel, smem));
+    dim3 grid(2 * ((m.n_tokens + 2 * tc::kTileM - 1) / (2 * tc::kTileM)), m.instances);
+    VSCAN_LAUNCH("assign_tensor", stream,
+                 (void)launch_dependent(tc::assign_pair_kernel, grid, dim3(tc::kThreads), smem, stream, map, map_b, p));
+    return VSCAN_OK;
   }
   const size_t smem = tc::smem_bytes(p);
   VSCAN_CUDA_TRY(allow_smem(tc::assign_tensor_kernel, smem));
@@ -709,7 +898,7 @@ vscan_status launch_merge_interleaved(const MergeParams& m_in, cudaStream_t stre
   tc::Params p; tc::Persist ps; size_t smem;
   if (!plan_persistent(m, p, ps, smem)) return VSCAN_ERR_UNSUPPORTED;
   CUtensorMap map, map_b;
-  vscan_status st = encode_maps(m, p, map, map_b);
+  vscan_status st = encode_maps(m, p, map, map_b, p.n_pad);
   if (st != VSCAN_OK) return st;
   {   // packed kept rows + their inverse norms; also clears the status word and the counters
     dim3 pgrid((static_cast<unsigned>(p.n_pad) + 7) / 8, m.instances);
