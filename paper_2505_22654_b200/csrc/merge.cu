@@ -415,6 +415,8 @@ static vscan_status validate_merge(const vscan_merge_desc* d) {
 
 // rows per instance of the packed copy of the kept rows: whole 256-row rounds for large kept sets, else
 // the kept count rounded up to the MMA's granularity of 16
+// kept sets above this size (at least four rounds of 256) are scanned in two shares by the CTA-pair assignment
+constexpr int kSplitKept = 768;
 static size_t packed_rows(int n_kept) { return n_kept > 256 ? round_up(n_kept, 256) : round_up(n_kept, 16); }
 
 extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
@@ -430,6 +432,10 @@ extern "C" size_t vscan_merge_workspace_bytes(const vscan_merge_desc* d) {
     const size_t md = d->metric ? d->metric_dim : d->dim;
     bytes += round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * md * 2, 256);
     bytes += round_up((static_cast<size_t>(d->instances) + 1) * sizeof(int), 256);   // counters of the persistent path
+    if (d->n_kept > kSplitKept) {   // the kept set is scanned in two shares: their partial results and the tiles' tickets
+      bytes += round_up(2 * static_cast<size_t>(d->instances) * d->n_tokens * sizeof(float2), 256);
+      bytes += round_up(static_cast<size_t>(d->instances) * ((d->n_tokens + 127) / 128) * sizeof(int), 256);
+    }
   }
   return bytes;
 }
@@ -467,6 +473,12 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
   p.counters = p.kept_packed ? reinterpret_cast<int*>(static_cast<char*>(p.kept_packed) +
                                                       round_up(static_cast<size_t>(d->instances) * packed_rows(d->n_kept) * p.metric_dim * 2, 256))
                              : nullptr;
+  p.partial = nullptr; p.tickets = nullptr;
+  if (p.counters && d->n_kept > kSplitKept) {
+    char* after = reinterpret_cast<char*>(p.counters) + round_up((static_cast<size_t>(d->instances) + 1) * sizeof(int), 256);
+    p.partial = reinterpret_cast<float2*>(after);
+    p.tickets = reinterpret_cast<int*>(after + round_up(2 * static_cast<size_t>(d->instances) * d->n_tokens * sizeof(float2), 256));
+  }
   p.merged = d->merged; p.counts = d->counts;
   p.instances = d->instances; p.row_len = d->row_len; p.cls_offset = d->cls_offset;
   p.n_tokens = d->n_tokens; p.dim = d->dim; p.n_kept = d->n_kept;

@@ -18,6 +18,8 @@ struct MergeParams {
   int* counters;        // [instances + 1] counters of the persistent path                              (workspace)
   int32_t* order;       // [instances][n_tokens] tokens ordered by slot, long instances only            (workspace)
   int32_t* order_start; // [instances][n_kept + 1] segment starts of `order`                            (workspace)
+  float2* partial;      // [2][instances][n_tokens] (value, slot) per share of the kept set, kept sets above 768 (workspace)
+  int* tickets;         // [instances][ceil(n_tokens / 128)] shares of a tile that have finished                  (workspace)
   int clear_status;     // this launch resets the status word (first launch of a call)
   uint32_t* status;     // device status word
   int instances, row_len, cls_offset, n_tokens, dim, metric_dim, n_kept;

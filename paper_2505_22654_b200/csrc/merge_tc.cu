@@ -274,31 +274,54 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
 // (a cluster of two, on the two SMs of one TPC) takes 256 tokens; each CTA loads its own 128 token rows and HALF of
 // the kept rows of a stage, and one MMA of M = 256 issued by the even CTA runs on both SMs, each tensor core reading
 // its own token tile and both halves of the kept rows.  Per 128 tokens and stage an SM takes in 16 KB + n_pad/2 rows
-// instead of 16 KB + n_pad rows, which is what bounds the single-CTA form at these sizes.
+// instead of 16 KB + n_pad rows.
+// The kernel is persistent: pair i works through items i, i + pairs, ...; an item is a 256-token tile and one of
+// `splits` contiguous shares of the n-chunks (two shares when there are at least four chunks, so that the number of
+// items divides well over the pairs).  The stage ring and the two accumulators run on across items.
 //   warp 0 (both CTAs)   producer: waits on its own `empty`, loads into its own shared memory, bytes counted on
 //                        the leader's `full` (armed by the leader's producer with the bytes of both CTAs)
 //   warp 1 (leader)      MMA issuer; after a stage's MMAs one commit per CTA frees the stage in both, after an
 //                        n-chunk one commit per CTA publishes the accumulator in both
 //   warps 2-5 (both)     read their CTA's 128 accumulator rows, running arg-max; the release of an accumulator is
-//                        an arrive on the leader's `tmem_empty` (count 8: four warps of each CTA)
+//                        an arrive on the leader's `tmem_empty` (count 8: four warps of each CTA).  With two shares
+//                        each leaves (value, slot) per token in the workspace and takes a ticket of its 128-token
+//                        tile; whoever comes last compares the two (equal values: the lower slot) and writes the
+//                        assignment.  Nobody waits for the other share.
 // Tensor memory is allocated and freed by warp 1 of both CTAs (pair-wide allocation); a cluster barrier before the
 // release makes sure neither CTA leaves, or frees anything, while the other may still use it.  Every mbarrier wait
 // is bounded as in assign_tile.
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads)
-assign_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p) {
+struct PairPlan {
+  int items, ptiles, splits, chunks_per_split;
+  float2* partial;    // [splits][instances][n_tokens] (value, slot as int bits), only with splits > 1
+  int* tickets;       // [instances][ceil(n_tokens / 128)], zero at launch
+};
+
+constexpr int kPairThreads = kThreads + 32;   // a second producer warp
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kPairThreads)
+assign_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, Params p, PairPlan pl) {
   extern __shared__ unsigned char smem_dyn[];
   __shared__ Shared sh;
+  __shared__ int ticket;
   unsigned char* tiles = smem_dyn + ((1024u - (static_cast<uint32_t>(__cvta_generic_to_shared(smem_dyn)) & 1023u)) & 1023u);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const MergeParams& m = p.m;
   const uint32_t rank = pair_rank();
   const bool leader = rank == 0;
-  const int b = blockIdx.y, t0 = (blockIdx.x >> 1) * (2 * kTileM) + static_cast<int>(rank) * kTileM;
+  const int pair = blockIdx.x >> 1, pairs = gridDim.x >> 1;
   volatile int* abort_flag = &sh.abort_flag;
   const int half_rows = p.n_pad / 2;                              // kept rows of a stage held by this CTA
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;      // b_stage_bytes: half_rows * 128, rounded to 1024
   float* inv_norm = reinterpret_cast<float*>(tiles + p.stages * stage_bytes);   // [accumulator][n_pad]
-  const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
+  const int per_instance = pl.splits * pl.ptiles;
+  // item -> instance, share of the n-chunks [c_lo, c_hi), first token of this CTA's 128 rows
+  auto decode = [&](int item, int& b, int& share, int& c_lo, int& c_hi, int& t0) {
+    b = item / per_instance;
+    const int rem = item - b * per_instance;
+    share = rem / pl.ptiles;
+    t0 = (rem - share * pl.ptiles) * (2 * kTileM) + static_cast<int>(rank) * kTileM;
+    c_lo = share * pl.chunks_per_split;
+    c_hi = min(p.n_chunks, c_lo + pl.chunks_per_split);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
@@ -316,58 +339,94 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_acc = sh.tmem_base;
   grid_dependency_launch();
-  grid_dependency_wait();   // kept list, packed rows and norms come from the kernels before this one; nothing is written before
-  if (m.clear_status && b == 0 && blockIdx.x == 0 && threadIdx.x == 0) *m.status = 0u;
+  grid_dependency_wait();   // kept list, packed rows, norms and zeroed tickets come from the kernels before this one; nothing is written before
+  if (m.clear_status && blockIdx.x == 0 && threadIdx.x == 0) *m.status = 0u;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------ producer
-    int it = 0;
+  if (warp == 0 || warp == 6) {
+    // ------------------------------------------------------------ producers: warp 0 the token tiles, warp 6 the kept rows
+    // (two warps, so that the two loads of a stage are issued side by side; the leader's warp 0 arms the barrier)
+    const bool loads_a = warp == 0;
+    int s = 0, it = 0;
+    uint32_t phase = 0;     // parity of the stage's current round
     bool ok = true;
-    for (int nc = 0; nc < p.n_chunks; ++nc) {
-      for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-        const int s = it % p.stages, round = it / p.stages;
-        if (ok && round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
-        if (!ok) continue;
-        if (lane == 0) {
-          unsigned char* at = tiles + s * stage_bytes;
-          if (leader) mbar_arrive_expect_tx(&sh.full[s], 2u * static_cast<uint32_t>(p.a_stage_bytes + half_rows * 128));
-          const uint32_t bar = pair_addr(&sh.full[s], 0);
-          pair_tma_load_3d(at, &map_a, bar, kc * kChunkK, m.cls_offset + t0, b);
-          pair_tma_load_3d(at + p.a_stage_bytes, &map_b, bar, kc * kChunkK, nc * p.n_pad + static_cast<int>(rank) * half_rows, b);
+    // The token tile of an item comes from DRAM the first time it is read (the later n-chunks find it in L2), and a
+    // stage is complete only when its last byte is there: the tile of the NEXT item is therefore asked into L2 while
+    // the first n-chunk of the current one streams through (lane 1; the very first tile up front by all lanes).
+    if (loads_a && pair < pl.items) {
+      int b, share, c_lo, c_hi, t0;
+      decode(pair, b, share, c_lo, c_hi, t0);
+      for (int kc = lane; kc < p.k_chunks; kc += 32) tma_prefetch_l2_3d(&map_a, kc * kChunkK, m.cls_offset + t0, b);
+    }
+    const uint32_t full0 = pair_addr(&sh.full[0], 0);   // the leader's `full` barriers, 8 bytes apart
+    for (int item = pair; item < pl.items; item += pairs) {
+      int b, share, c_lo, c_hi, t0;
+      decode(item, b, share, c_lo, c_hi, t0);
+      int nb = 0, nshare, nc_lo, nc_hi, nt0 = 0;
+      const bool has_next = loads_a && item + pairs < pl.items;
+      if (has_next) decode(item + pairs, nb, nshare, nc_lo, nc_hi, nt0);
+      for (int nc = c_lo; nc < c_hi; ++nc) {
+        const int b_row = nc * p.n_pad + static_cast<int>(rank) * half_rows;
+        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
+          if (ok && it >= p.stages) ok = mbar_wait_warp(&sh.empty[s], phase ^ 1u, abort_flag);
+          if (ok) {
+            if (lane == 1 && has_next && nc == c_lo) tma_prefetch_l2_3d(&map_a, kc * kChunkK, m.cls_offset + nt0, nb);
+            if (lane == 0) {
+              unsigned char* at = tiles + s * stage_bytes;
+              const uint32_t bar = full0 + 8u * s;
+              if (loads_a) {
+                if (leader) mbar_arrive_expect_tx(&sh.full[s], 2u * static_cast<uint32_t>(p.a_stage_bytes + half_rows * 128));
+                pair_tma_load_3d(at, &map_a, bar, kc * kChunkK, m.cls_offset + t0, b);
+              } else {
+                pair_tma_load_3d(at + p.a_stage_bytes, &map_b, bar, kc * kChunkK, b_row, b);
+              }
+            }
+          }
+          if (++s == p.stages) { s = 0; phase ^= 1u; }
         }
       }
     }
     // the leader's commits to this CTA's `empty` barriers have all arrived before its shared memory goes
-    for (int i = max(0, it - p.stages); i < it; ++i)
-      if (ok) ok = mbar_wait_warp(&sh.empty[i % p.stages], (i / p.stages) & 1, abort_flag);
+    for (int i = 0; i < min(it, p.stages); ++i) {
+      if (s == 0) { s = p.stages; phase ^= 1u; }
+      --s;
+      if (ok) ok = mbar_wait_warp(&sh.empty[s], phase, abort_flag);
+    }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (leader only)
     if (leader && lane == 0) {
       const uint32_t idesc = pair_instr_desc_bf16(p.n_pad);
-      int it = 0;
-      for (int nc = 0; nc < p.n_chunks && !*abort_flag; ++nc) {
-        const int acc = nc & 1, use = nc >> 1;
-        if (use > 0) {
-          if (!mbar_wait(&sh.tmem_empty[acc], (use - 1) & 1, abort_flag)) break;
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        }
-        const uint32_t d_addr = tmem_acc + acc * p.n_pad;
-        bool ok = true;
-        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-          const int s = it % p.stages, round = it / p.stages;
-          if (!mbar_wait(&sh.full[s], round & 1, abort_flag)) { ok = false; break; }
-          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = smem_u32(tiles + s * stage_bytes), b_addr = a_addr + p.a_stage_bytes;
-          const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
+      int s = 0, g = 0;      // stage of the ring; n-chunks since the start of the kernel
+      uint32_t phase = 0;
+      bool ok = true;
+      const uint32_t tiles_addr = smem_u32(tiles);
+      const uint32_t empty_local = smem_u32(&sh.empty[0]), empty_peer = pair_addr(&sh.empty[0], 1);
+      for (int item = pair; item < pl.items && ok; item += pairs) {
+        int b, share, c_lo, c_hi, t0;
+        decode(item, b, share, c_lo, c_hi, t0);
+        for (int nc = c_lo; nc < c_hi && ok && !*abort_flag; ++nc, ++g) {
+          const int acc = g & 1, use = g >> 1;
+          if (use > 0) {
+            if (!mbar_wait(&sh.tmem_empty[acc], (use - 1) & 1, abort_flag)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          }
+          const uint32_t d_addr = tmem_acc + acc * p.n_pad;
+          for (int kc = 0; kc < p.k_chunks; ++kc) {
+            if (!mbar_wait(&sh.full[s], phase, abort_flag)) { ok = false; break; }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_addr = tiles_addr + s * stage_bytes, b_addr = a_addr + p.a_stage_bytes;
+            const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
 #pragma unroll
-          for (int k = 0; k < kChunkK / 16; ++k)
-            pair_umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
-          pair_umma_commit(smem_u32(&sh.empty[s]));
-          pair_umma_commit(pair_addr(&sh.empty[s], 1));
+            for (int k = 0; k < kChunkK / 16; ++k)
+              pair_umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
+            pair_umma_commit(empty_local + 8u * s);
+            pair_umma_commit(empty_peer + 8u * s);
+            if (++s == p.stages) { s = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          pair_umma_commit(smem_u32(&sh.tmem_full[acc]));
+          pair_umma_commit(pair_addr(&sh.tmem_full[acc], 1));
         }
-        if (!ok) break;
-        pair_umma_commit(smem_u32(&sh.tmem_full[acc]));
-        pair_umma_commit(pair_addr(&sh.tmem_full[acc], 1));
+        if (*abort_flag) ok = false;
       }
     }
     __syncwarp();
@@ -376,55 +435,90 @@ assign_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const int ptid = (warp - 2) * 32 + lane;
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    float best_val = -INFINITY;
-    int best_idx = 0;
+    const int tiles128 = (m.n_tokens + kTileM - 1) / kTileM;
     bool ok = true;
-    for (int nc = 0; nc < p.n_chunks; ++nc) {
-      const int n0 = nc * p.n_pad, acc = nc & 1, use = nc >> 1;
+    int g = 0;
+    // Once `ok` drops the loops keep running with their work skipped, so that the four warps execute the same
+    // sequence of named barriers whatever happens.
+    for (int item = pair; item < pl.items; item += pairs) {
+      int b, share, c_lo, c_hi, t0;
+      decode(item, b, share, c_lo, c_hi, t0);
+      const int32_t* kept = m.kept + static_cast<size_t>(b) * m.n_kept;
+      float best_val = -INFINITY;
+      int best_idx = 0;
+      for (int nc = c_lo; nc < c_hi; ++nc, ++g) {
+        const int n0 = nc * p.n_pad, acc = g & 1, use = g >> 1;
 #pragma unroll
-      for (int u = 0; u < 2; ++u) {
-        const int r = ptid + 128 * u;
-        if (r < p.n_pad)
-          inv_norm[acc * p.n_pad + r] = n0 + r < m.n_kept ? __ldcg(m.inv_norm + static_cast<size_t>(b) * m.n_kept + n0 + r) : 0.f;
-      }
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
-      if (!ok) continue;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.n_pad;
-      for (int c0 = 0; c0 < p.n_pad; c0 += 32) {
-        uint32_t v[32];
-        if (p.n_pad - c0 >= 32) tmem_ld32(taddr + c0, v);
-        else {
-          tmem_ld16(taddr + c0, v);
-#pragma unroll
-          for (int j = 16; j < 32; ++j) v[j] = 0u;
+        for (int u = 0; u < 2; ++u) {
+          const int r = ptid + 128 * u;
+          if (r < p.n_pad)
+            inv_norm[acc * p.n_pad + r] = n0 + r < m.n_kept ? __ldcg(m.inv_norm + static_cast<size_t>(b) * m.n_kept + n0 + r) : 0.f;
         }
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
+        if (!ok) continue;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * p.n_pad;
+        for (int c0 = 0; c0 < p.n_pad; c0 += 32) {
+          uint32_t v[32];
+          if (p.n_pad - c0 >= 32) tmem_ld32(taddr + c0, v);
+          else {
+            tmem_ld16(taddr + c0, v);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int s_idx = n0 + c0 + j;
-          if (c0 + j < p.n_pad && s_idx < m.n_kept) {
-            const float val = __uint_as_float(v[j]) * inv_norm[acc * p.n_pad + c0 + j];
-            if (val > best_val) { best_val = val; best_idx = s_idx; }
+            for (int j = 16; j < 32; ++j) v[j] = 0u;
+          }
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int s_idx = n0 + c0 + j;
+            if (c0 + j < p.n_pad && s_idx < m.n_kept) {
+              const float val = __uint_as_float(v[j]) * inv_norm[acc * p.n_pad + c0 + j];
+              if (val > best_val) { best_val = val; best_idx = s_idx; }
+            }
+          }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          if (leader) mbar_arrive(&sh.tmem_empty[acc]);
+          else pair_remote_arrive(pair_addr(&sh.tmem_empty[acc], 0));
+        }
+      }
+      // ---- the item's result for token t0 + row is (best_val, best_idx)
+      bool write = ok;
+      if (pl.splits > 1) {
+        const size_t inst_tokens = static_cast<size_t>(m.instances) * m.n_tokens;
+        const size_t tok = static_cast<size_t>(b) * m.n_tokens + t0 + row;
+        if (ok && t0 + row < m.n_tokens) pl.partial[share * inst_tokens + tok] = make_float2(best_val, __int_as_float(best_idx));
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (ptid == 0) ticket = (ok && t0 < m.n_tokens) ? atomicAdd(&pl.tickets[b * tiles128 + t0 / kTileM], 1) : -1;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        write = ticket == pl.splits - 1;          // the last share of this tile to finish combines them
+        if (write) {
+          __threadfence();
+          if (t0 + row < m.n_tokens) {
+            for (int h2 = 0; h2 < pl.splits; ++h2) {
+              if (h2 == share) continue;
+              const float2 o = __ldcg(pl.partial + h2 * inst_tokens + tok);
+              const int oi = __float_as_int(o.y);
+              if (o.x > best_val || (o.x == best_val && oi < best_idx)) { best_val = o.x; best_idx = oi; }
+            }
           }
         }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) {
-        if (leader) mbar_arrive(&sh.tmem_empty[acc]);
-        else pair_remote_arrive(pair_addr(&sh.tmem_empty[acc], 0));
+      sh.best_slot[row] = best_idx;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (write) {
+        for (int s_idx = ptid; s_idx < m.n_kept; s_idx += 128) {   // a kept token belongs to its own slot
+          const int t = min(max(kept[s_idx], 0), m.n_tokens - 1);
+          if (t >= t0 && t < t0 + kTileM) sh.best_slot[t - t0] = s_idx;
+        }
       }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (write && t0 + ptid < m.n_tokens) m.assign[static_cast<size_t>(b) * m.n_tokens + t0 + ptid] = sh.best_slot[ptid];
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // best_slot and ticket are reused by the next item
     }
-    sh.best_slot[row] = best_idx;
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    for (int s_idx = ptid; s_idx < m.n_kept; s_idx += 128) {   // a kept token belongs to its own slot
-      const int t = min(max(kept[s_idx], 0), m.n_tokens - 1);
-      if (t >= t0 && t < t0 + kTileM) sh.best_slot[t - t0] = s_idx;
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (ok && t0 + ptid < m.n_tokens) m.assign[static_cast<size_t>(b) * m.n_tokens + t0 + ptid] = sh.best_slot[ptid];
   }
 
   // ------------------------------------------------------------ teardown
@@ -491,6 +585,8 @@ __global__ void __launch_bounds__(256) pack_kept_norm_kernel(MergeParams m, int 
   if (blockIdx.x == 0 && blockIdx.y == 0) {
     if (threadIdx.x == 0) *m.status = 0u;
     for (int i = threadIdx.x; i <= m.instances; i += 256) m.counters[i] = 0;
+    if (m.tickets)
+      for (int i = threadIdx.x; i < m.instances * ((m.n_tokens + kTileM - 1) / kTileM); i += 256) m.tickets[i] = 0;
   }
   const int b = blockIdx.y, s = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (s >= rows_packed) return;
@@ -814,6 +910,16 @@ static vscan_status encode_maps(const MergeParams& m, const tc::Params& p, CUten
   return r == CUDA_SUCCESS ? VSCAN_OK : VSCAN_ERR_UNSUPPORTED;
 }
 
+static int sm_count() {
+  static int n = 0;
+  if (n == 0) {
+    int dev = 0, v = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+    else return 148;
+  }
+  return n;
+}
+
 vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   tc::Params p;
   if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
@@ -821,6 +927,7 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   const bool pair = p.b_packed && p.norms_given && p.n_pad % 16 == 0;
   if (pair) {
     p.b_stage_bytes = ((p.n_pad / 2 * tc::kChunkK * 2) + 1023) / 1024 * 1024;
+    // (a seventh stage, which just fits, measured slower: 301 us against 294 us at 2048 kept tokens)
     int stages = (215 * 1024) / (p.a_stage_bytes + p.b_stage_bytes);
     p.stages = stages > tc::kMaxStages ? tc::kMaxStages : stages;
   }
@@ -833,11 +940,20 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
                  (void)launch_dependent(tc::pack_kept_norm_kernel, pgrid, dim3(256), 0, stream, m, p.n_chunks * p.n_pad));
   }
   if (pair) {
+    tc::PairPlan pl;
+    pl.ptiles = (m.n_tokens + 2 * tc::kTileM - 1) / (2 * tc::kTileM);
+    pl.splits = (p.n_chunks >= 4 && m.partial && m.tickets) ? 2 : 1;
+    pl.chunks_per_split = (p.n_chunks + pl.splits - 1) / pl.splits;
+    pl.partial = m.partial; pl.tickets = m.tickets;
+    const long long items = 1ll * m.instances * pl.splits * pl.ptiles;
+    if (items > 0x3fffffffLL) return VSCAN_ERR_UNSUPPORTED;
+    pl.items = static_cast<int>(items);
     const size_t smem = tc::smem_bytes(p);
     VSCAN_CUDA_TRY(allow_smem(tc::assign_pair_kernel, smem));
-    dim3 grid(2 * ((m.n_tokens + 2 * tc::kTileM - 1) / (2 * tc::kTileM)), m.instances);
+    const int pairs_max = sm_count() / 2;
+    const unsigned pairs = static_cast<unsigned>(pl.items < pairs_max ? pl.items : pairs_max);
     VSCAN_LAUNCH("assign_tensor", stream,
-                 (void)launch_dependent(tc::assign_pair_kernel, grid, dim3(tc::kThreads), smem, stream, map, map_b, p));
+                 (void)launch_dependent(tc::assign_pair_kernel, dim3(2 * pairs), dim3(tc::kPairThreads), smem, stream, map, map_b, p, pl));
     return VSCAN_OK;
   }
   const size_t smem = tc::smem_bytes(p);
@@ -849,16 +965,6 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
 }
 
 // ---- assignment + group means in one persistent launch
-static int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0, v = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
-    else return 148;
-  }
-  return n;
-}
-
 static bool plan_persistent(const MergeParams& m, tc::Params& p, tc::Persist& ps, size_t& smem) {
   if (!tc::plan(m, p) || p.n_chunks != 1 || p.b_packed || m.kept_packed == nullptr) return false;
   p.b_packed = 1;   // one producer warp per SM: a tile load of the packed kept rows per stage instead of n_pad / 4 row gathers

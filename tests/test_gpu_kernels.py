@@ -170,12 +170,13 @@ def test_merge_exact_ties_and_duplicates():
 
 
 @pytest.mark.parametrize("N,D,K1,c", [(576, 1024, 64, 1), (576, 1024, 192, 1), (300, 72, 17, 0), (130, 264, 130, 1),
-                                      (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0)])
+                                      (1000, 1280, 300, 0), (128, 64, 1, 1), (129, 128, 16, 0),
+                                      (1500, 256, 800, 1), (1300, 128, 1100, 0)])
 @pytest.mark.parametrize("path", ["tensor", "interleaved"])
 def test_merge_tensor_path_matches_oracle(N, D, K1, c, path):
     """The tcgen05 path on its own (path = TENSOR): tile tails, kept counts that are not multiples of
-    16, more than 256 kept tokens (several accumulator rounds), feature dims that are not multiples
-    of 64."""
+    16, more than 256 kept tokens (several accumulator rounds on CTA pairs), more than 768 (the kept set scanned in
+    two shares whose results are combined by whichever finishes last), feature dims that are not multiples of 64."""
     cfg = small_cfg("bf16", grid_h=1, grid_w=N, win_h=1, win_w=N, k_w=0, k_g=K1, D=D, C=1, B=2, cls=c)
     x = round_to_dtype(RNG.standard_normal((2, N + c, D)).astype(np.float32), "bf16")
     kept = np.stack([np.sort(RNG.choice(N, K1, replace=False)) for _ in range(2)])
