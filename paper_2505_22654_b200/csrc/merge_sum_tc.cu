@@ -116,27 +116,29 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
     // ------------------------------------------------------------ producer (the features are an input of the call:
     // their loads need not wait for the kernel before this one)
     bool ok = true;
-    int it = 0;
+    int s = 0, it = 0;       // ring position as counters: no division per tile
+    uint32_t phase = 0;
     for (int w = blockIdx.x; w < p.items && ok; w += gridDim.x) {
       const int b = w / p.slices, col0 = (w - b * p.slices) * p.m_tiles * 128;
       const int boxes = min(p.m_tiles, (m.dim - col0) / 128) * 2;
       for (int t = 0; t < p.tiles && ok; ++t, ++it) {
-        const int s = it % p.stages, round = it / p.stages;
-        if (round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
+        if (it >= p.stages) ok = mbar_wait_warp(&sh.empty[s], phase ^ 1u, abort_flag);
         if (!ok) break;
-        if (lane == 0) {
-          unsigned char* st = base + s * stage_bytes;
-          mbar_arrive_expect_tx(&sh.full[s], boxes * kBoxBytes);
-          for (int i = 0; i < boxes; ++i)
-            tma_load_3d(st + i * kBoxBytes, &map_x, &sh.full[s], col0 + i * 64, m.cls_offset + t * kTileTokens, b);
-        }
+        unsigned char* st = base + s * stage_bytes;
+        if (lane == 0) mbar_arrive_expect_tx(&sh.full[s], boxes * kBoxBytes);
+        __syncwarp();
+        if (lane < boxes)    // one box per lane, issued by one instruction
+          tma_load_3d(st + lane * kBoxBytes, &map_x, &sh.full[s], col0 + lane * 64, m.cls_offset + t * kTileTokens, b);
+        if (++s == p.stages) { s = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = true;
-      int it = 0, i = 0;
+      int it = 0, i = 0, s = 0;
+      uint32_t phase = 0;
+      const uint32_t base_addr = smem_u32(base), onehot_addr = smem_u32(onehot);
       for (int w = blockIdx.x; w < p.items && ok && !*abort_flag; w += gridDim.x, ++i) {
         const int b = w / p.slices, col0 = (w - b * p.slices) * p.m_tiles * 128;
         const int my_tiles = min(p.m_tiles, (m.dim - col0) / 128);
@@ -147,11 +149,11 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         }
         for (int t = 0; t < p.tiles; ++t, ++it) {
-          const int s = it % p.stages, round = it / p.stages, pb = it % kOneHots;
-          if (!mbar_wait(&sh.full[s], round & 1, abort_flag) || !mbar_wait(&sh.p_full[pb], (it / kOneHots) & 1, abort_flag)) { ok = false; break; }
+          const int pb = it % kOneHots;
+          if (!mbar_wait(&sh.full[s], phase, abort_flag) || !mbar_wait(&sh.p_full[pb], (it / kOneHots) & 1, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t st_addr = smem_u32(base + s * stage_bytes);
-          const uint64_t da = smem_desc_sw128(smem_u32(onehot + pb * onehot_bytes));
+          const uint32_t st_addr = base_addr + s * stage_bytes;
+          const uint64_t da = smem_desc_sw128(onehot_addr + pb * onehot_bytes);
 #pragma unroll
           for (int k = 0; k < kTileTokens / 16; ++k) {   // 16 tokens = 32 bytes of a one-hot row, two 1024-byte groups of the token tile
             const uint64_t db = smem_desc_mn_sw128(st_addr + k * 2048, kBoxBytes);
@@ -159,6 +161,7 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
           }
           umma_commit(&sh.empty[s]);
           umma_commit(&sh.p_empty[pb]);
+          if (++s == p.stages) { s = 0; phase ^= 1u; }
         }
         if (ok) umma_commit(&sh.acc_full[acc]);
       }

@@ -94,7 +94,8 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
     const int groups = p.n_pad / 4;                 // gathers per stage
     const int row_base = b * m.row_len + m.cls_offset;
     const int first = row_base + min(max(kept[0], 0), m.n_tokens - 1);
-    int it = 0;
+    int s = 0, it = 0;      // ring position kept as counters: no division per stage
+    uint32_t phase = 0;
     bool ok = true;
     for (int nc = 0; nc < p.n_chunks; ++nc) {
       int rows[2][4];
@@ -108,29 +109,32 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
         }
       }
       for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-        const int s = it % p.stages, round = it / p.stages;
-        if (ok && round > 0) ok = mbar_wait_warp(&sh.empty[s], (round - 1) & 1, abort_flag);
-        if (!ok) continue;
-        unsigned char* at = tiles + s * stage_bytes;
-        if (lane == 0) {
-          mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes + p.n_pad * 128);
-          tma_load_3d(at, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
-          if (p.b_packed) tma_load_3d(at + p.a_stage_bytes, &map_b, &sh.full[s], kc * kChunkK, nc * p.n_pad, b);
-        }
+        if (ok && it >= p.stages) ok = mbar_wait_warp(&sh.empty[s], phase ^ 1u, abort_flag);
+        if (ok) {
+          unsigned char* at = tiles + s * stage_bytes;
+          if (lane == 0) {
+            mbar_arrive_expect_tx(&sh.full[s], p.a_stage_bytes + p.n_pad * 128);
+            tma_load_3d(at, &map_a, &sh.full[s], kc * kChunkK, m.cls_offset + t0, b);
+            if (p.b_packed) tma_load_3d(at + p.a_stage_bytes, &map_b, &sh.full[s], kc * kChunkK, nc * p.n_pad, b);
+          }
 #pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int g = lane + 32 * i;
-          if (g < groups && !p.b_packed)
-            tma_gather4(at + p.a_stage_bytes + g * 512, &map_b, &sh.full[s], kc * kChunkK, rows[i][0], rows[i][1],
-                        rows[i][2], rows[i][3]);
+          for (int i = 0; i < 2; ++i) {
+            const int g = lane + 32 * i;
+            if (g < groups && !p.b_packed)
+              tma_gather4(at + p.a_stage_bytes + g * 512, &map_b, &sh.full[s], kc * kChunkK, rows[i][0], rows[i][1],
+                          rows[i][2], rows[i][3]);
+          }
         }
+        if (++s == p.stages) { s = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = instr_desc_bf16(p.n_pad);
-      int it = 0;
+      int s = 0;
+      uint32_t phase = 0;
+      const uint32_t tiles_addr = smem_u32(tiles);
       for (int nc = 0; nc < p.n_chunks && !*abort_flag; ++nc) {
         const int acc = nc & 1, use = nc >> 1;
         if (use > 0) {
@@ -139,16 +143,16 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
         }
         const uint32_t d_addr = tmem_acc + acc * p.n_pad;
         bool ok = true;
-        for (int kc = 0; kc < p.k_chunks; ++kc, ++it) {
-          const int s = it % p.stages, round = it / p.stages;
-          if (!mbar_wait(&sh.full[s], round & 1, abort_flag)) { ok = false; break; }
+        for (int kc = 0; kc < p.k_chunks; ++kc) {
+          if (!mbar_wait(&sh.full[s], phase, abort_flag)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = smem_u32(tiles + s * stage_bytes), b_addr = a_addr + p.a_stage_bytes;
+          const uint32_t a_addr = tiles_addr + s * stage_bytes, b_addr = a_addr + p.a_stage_bytes;
           const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(b_addr);
 #pragma unroll
           for (int k = 0; k < kChunkK / 16; ++k)   // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
             umma_bf16(d_addr, da + 2u * k, db + 2u * k, idesc, kc > 0 || k > 0);
           umma_commit(&sh.empty[s]);
+          if (++s == p.stages) { s = 0; phase ^= 1u; }
         }
         if (!ok) break;
         umma_commit(&sh.tmem_full[acc]);
@@ -162,7 +166,8 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
     const int row = quarter * 32 + lane;      // token row of this thread within the tile
     float best_val = -INFINITY;
     int best_idx = 0;
-    int it = 0;
+    int s = 0;
+    uint32_t phase = 0;
     bool ok = true;
     // Once `ok` drops the loop keeps running with its work skipped, so that the four warps execute
     // the same sequence of named barriers and warp-wide instructions whatever happens.
@@ -171,11 +176,12 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
       // |m_s|^2 of the kept rows of this n-chunk, accumulated from the B stages as they pass through
       // shared memory (thread ptid owns rows ptid and ptid + 128)
       float ss[2] = {0.f, 0.f};
-      for (int kc = 0; kc < (p.norms_given ? 0 : p.k_chunks); ++kc, ++it) {
-        const int s = it % p.stages, round = it / p.stages;
-        if (ok) ok = mbar_wait_warp(&sh.full[s], round & 1, abort_flag);
+      for (int kc = 0; kc < (p.norms_given ? 0 : p.k_chunks); ++kc) {
+        const int cur = s;
+        if (ok) ok = mbar_wait_warp(&sh.full[cur], phase, abort_flag);
+        if (++s == p.stages) { s = 0; phase ^= 1u; }
         if (!ok) continue;
-        const unsigned char* bt = tiles + s * stage_bytes + p.a_stage_bytes;
+        const unsigned char* bt = tiles + cur * stage_bytes + p.a_stage_bytes;
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           const int r = ptid + 128 * u;
@@ -190,7 +196,7 @@ __device__ __forceinline__ void assign_tile(const CUtensorMap* map_a_ptr, const 
           }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sh.empty[s]);
+        if (lane == 0) mbar_arrive(&sh.empty[cur]);
       }
       // the buffer was last read two chunks ago, before that chunk's arrive on tmem_empty
 #pragma unroll
