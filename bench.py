@@ -69,6 +69,18 @@ def measured_peaks() -> tuple[float, str]:
         return FALLBACK_HBM_GBS, "fallback"
 
 
+FALLBACK_BF16_TFLOPS_SUSTAINED = 1400.0   # an earlier measurement on this machine, used when the measured file is absent
+
+
+def measured_tensor_peak() -> tuple[float, str]:
+    """Dense bf16 TFLOP/s of a library matrix product timed inside a long loop (the figure for a kernel that is
+    timed inside a step)."""
+    try:
+        return float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS_SUSTAINED, "fallback"
+
+
 # ------------------------------------------------------------------ clocks during the timed region
 class ClockSampler(threading.Thread):
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
@@ -363,11 +375,22 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
         achieved = dom_bytes / (kernels[dominant]["avg_us"] * 1e-6) / 1e9
         traffic = None
         try:
-            traffic = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json"))).get(dominant)
+            traffic = json.load(open(os.path.join(ROOT, "profiles", "dram_traffic.json"))).get(cfg.name, {}).get(dominant)
         except Exception:
             pass
         cpu = time_oracle(cfg) if (world == 1 and with_cpu and not args.no_cpu_baseline) else None
         step_gbs = alg["step"] / (ms_step * 1e-3) / 1e9
+        roof = {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
+                "algorithmic_bytes_per_launch": dom_bytes}
+        peak_tf, tf_kind = measured_tensor_peak()
+        if dominant in ("assign_tensor", "merge_persistent") and \
+                merge_flops(cfg) / (peak_tf * 1e12) > dom_bytes / (peak * 1e9):
+            # the similarity contraction takes longer at the tensor peak than its bytes at the HBM peak: a contraction
+            tf = merge_flops(cfg) / (kernels[dominant]["avg_us"] * 1e-6) / 1e12
+            roof = {"kernel": dominant, "bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s",
+                    "frac": tf / peak_tf, "traffic": traffic, "peak_kind": f"of {tf_kind} (bf16, sustained)",
+                    "algorithmic_flops_per_launch": merge_flops(cfg)}
         line = {
             "metric": METRIC, "value": world * cfg.B * args.steps / (ms_total * 1e-3), "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": ms_step,
@@ -381,9 +404,7 @@ def measure(args, cfg, rank, world, local_rank, dist, with_e2e=True, with_cpu=Tr
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "step_hbm": {"algorithmic_bytes": alg["step"], "achieved_gbs": step_gbs, "frac": step_gbs / peak,
                          "peak_gbs": peak, "peak_kind": peak_kind},
-            "roofline": {"kernel": dominant, "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": traffic, "peak_kind": f"of {peak_kind}",
-                         "algorithmic_bytes_per_launch": dom_bytes},
+            "roofline": roof,
             "kernels": kernels,
             "merge": {"flops_per_step": merge_flops(cfg),
                       "us": sum(kernels[n]["avg_us"] * kernels[n]["launches_per_step"] for n in merge_names),
