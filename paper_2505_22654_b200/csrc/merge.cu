@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kSlotsPerCta * 32) group_mean_kernel(MergePara
   extern __shared__ __align__(16) uint32_t list[];
   __shared__ int warp_sums[33];
   grid_dependency_wait();   // the assignments come from the kernel before this one
-  group_mean_body<T, VPL, R, kSlotsPerCta, kSlotsPerCta>(p, blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums,
+  group_mean_body<T, VPL, R, kSlotsPerCta, kSlotsPerCta>(p, gridDim.y - 1 - blockIdx.y, blockIdx.x * kSlotsPerCta, list, warp_sums,
                                                          static_cast<int>(threadIdx.x), CtaSync());
 }
 
@@ -163,7 +163,7 @@ template <typename T, int VPL, int R>
 __global__ void __launch_bounds__(128) group_mean_bits_kernel(MergeParams p) {
   extern __shared__ __align__(16) unsigned char smem_bits[];
   grid_dependency_wait();   // the assignments come from the kernel before this one
-  group_mean_bits_body<T, VPL, R>(p, blockIdx.y, blockIdx.x * 4, smem_bits);
+  group_mean_bits_body<T, VPL, R>(p, gridDim.y - 1 - blockIdx.y, blockIdx.x * 4, smem_bits);
 }
 
 // ---- long instances (more than 2048 tokens): members by counting sort, segments put in order, then the sums.
@@ -257,7 +257,7 @@ template <typename T, int VPL, int R>
 __global__ void __launch_bounds__(256) group_mean_sorted_kernel(MergeParams p, const int32_t* order, const int32_t* start, int chunks) {
   constexpr int E = Vec16<T>::kElems;
   grid_dependency_wait();
-  const int b = blockIdx.y, lane = threadIdx.x & 31;
+  const int b = gridDim.y - 1 - blockIdx.y, lane = threadIdx.x & 31;   // last instance first: the assignment pass has just read it
   const int task = blockIdx.x * 8 + (threadIdx.x >> 5);
   const int s = task / chunks, v0 = (task - s * chunks) * 32 * VPL;
   if (s >= p.n_kept) return;

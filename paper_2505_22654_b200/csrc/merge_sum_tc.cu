@@ -115,11 +115,13 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
   if (warp == 0) {
     // ------------------------------------------------------------ producer (the features are an input of the call:
     // their loads need not wait for the kernel before this one)
+    // Items run from the LAST instance to the first: the assignment pass before this kernel read the instances in
+    // ascending order, so the last ones are the part of the features that is still in L2.
     bool ok = true;
     int s = 0, it = 0;       // ring position as counters: no division per tile
     uint32_t phase = 0;
     for (int w = blockIdx.x; w < p.items && ok; w += gridDim.x) {
-      const int b = w / p.slices, col0 = (w - b * p.slices) * p.m_tiles * 128;
+      const int b = m.instances - 1 - w / p.slices, col0 = (w - (w / p.slices) * p.slices) * p.m_tiles * 128;
       const int boxes = min(p.m_tiles, (m.dim - col0) / 128) * 2;
       for (int t = 0; t < p.tiles && ok; ++t, ++it) {
         if (it >= p.stages) ok = mbar_wait_warp(&sh.empty[s], phase ^ 1u, abort_flag);
@@ -140,7 +142,7 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
       uint32_t phase = 0;
       const uint32_t base_addr = smem_u32(base), onehot_addr = smem_u32(onehot);
       for (int w = blockIdx.x; w < p.items && ok && !*abort_flag; w += gridDim.x, ++i) {
-        const int b = w / p.slices, col0 = (w - b * p.slices) * p.m_tiles * 128;
+        const int b = m.instances - 1 - w / p.slices, col0 = (w - (w / p.slices) * p.slices) * p.m_tiles * 128;
         const int my_tiles = min(p.m_tiles, (m.dim - col0) / 128);
         const uint32_t idesc = instr_desc_bf16_bmn(p.n_pad, my_tiles * 128);
         const int acc = i & 1, use = i >> 1;
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
     auto load = [&](int ww, int tt, int& a0, int& a1) {
       a0 = -1; a1 = -1;
       if (ww >= p.items) return;
-      const int32_t* ag = m.assign + static_cast<size_t>(ww / p.slices) * m.n_tokens;
+      const int32_t* ag = m.assign + static_cast<size_t>(m.instances - 1 - ww / p.slices) * m.n_tokens;
       const int tok0 = tt * kTileTokens + lane, tok1 = tok0 + 32;
       if (tok0 < m.n_tokens) a0 = __ldcg(ag + tok0);   // raw values: nothing here waits for the loads
       if (tok1 < m.n_tokens) a1 = __ldcg(ag + tok1);
@@ -225,7 +227,7 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
     bool ok = true;
     int i = 0;
     for (int w = blockIdx.x; w < p.items; w += gridDim.x, ++i) {
-      const int b = w / p.slices, slice = w - b * p.slices, col0 = slice * p.m_tiles * 128;
+      const int b = m.instances - 1 - w / p.slices, slice = w - (w / p.slices) * p.slices, col0 = slice * p.m_tiles * 128;
       const int my_tiles = min(p.m_tiles, (m.dim - col0) / 128);
       const int acc = i & 1;
       if (ok) ok = mbar_wait_warp(&sh.acc_full[acc], (i >> 1) & 1, abort_flag);
