@@ -95,35 +95,47 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(CompactParams 
   compact_row<kCompactThreads>(p, blockIdx.x, blockIdx.y);
 }
 
-// Score, top-k and compaction of Stage 2 in ONE launch.  The first n_score CTAs are the (head,
-// sequence) scoring CTAs of qk_softmax_role; the CTAs after them each move one output row.  Rows of
-// the system and text spans do not depend on the selection and are moved at once (they come first
-// in block order); a row of the visual span waits, with a bound, until the scoring CTA that finished
-// its sequence last has published the survivor list.  Blocks are dispatched in index order, so
-// every scoring CTA is running or done before a waiting CTA can occupy a slot.
+// Score, top-k and compaction of Stage 2 in ONE launch.  n_score CTAs are the (head, sequence)
+// scoring CTAs of qk_softmax_role; the others each move one output row.  Rows of the system and text
+// spans do not depend on the selection: they come first in block order, interleaved with the scoring
+// CTAs; a row of the visual span waits, with a bound, until the scoring CTA that finished its
+// sequence last has published the survivor list.  Blocks are dispatched in index order and every
+// scoring CTA has a lower index than any waiting CTA, so every scoring CTA is running or done
+// before a waiting CTA can occupy a slot.
 constexpr int kPruneThreads = 128;
 constexpr unsigned kReadySpinLimit = 1u << 22;
 
 template <typename T, int VPS>
 __global__ void __launch_bounds__(kPruneThreads, 8) prune_fused_kernel(QkParams q, CompactParams c, int n_score) {
   extern __shared__ __align__(16) float smem_f[];
-  const int blk = blockIdx.x;
-  if (blk < n_score) {
-    const int unit = blk / q.nsplit;   // (sequence, head), heads fastest; the shares of a unit are neighbours
-    qk_softmax_role<T, VPS>(q, unit % q.q_heads, unit / q.q_heads, smem_f, blk - unit * q.nsplit);
-    return;
-  }
-  int idx = blk - n_score;
+  // Block order: the scoring CTAs and the rows that do not depend on the selection are dealt out together, one
+  // scoring CTA per `period` blocks (scoring is bound by latency, the row copies by bandwidth: side by side they
+  // keep the memory pipe busy from the start); the rows that wait for a survivor list come after all of them.
   const int fixed_rows = c.seq_out - c.k_keep;           // system + text rows per sequence
+  const int n_fixed = c.batch * fixed_rows, n_indep = n_score + n_fixed;
+  const int blk = blockIdx.x;
+  int idx;                                                // row index: first the independent rows, then the dependent ones
+  if (blk < n_indep) {
+    const int period = n_score > 0 ? n_indep / n_score : 1;
+    const int qd = blk / period, rm = blk - qd * period;
+    if (qd < n_score && rm == 0) {
+      const int unit = qd / q.nsplit;   // (sequence, head), heads fastest; the shares of a unit are neighbours
+      qk_softmax_role<T, VPS>(q, unit % q.q_heads, unit / q.q_heads, smem_f, qd - unit * q.nsplit);
+      return;
+    }
+    idx = qd < n_score ? qd * (period - 1) + (rm - 1) : n_score * (period - 1) + (blk - n_score * period);
+  } else {
+    idx = blk - n_score;
+  }
   int r, b;
   bool dependent;
-  if (idx < c.batch * fixed_rows) {
+  if (idx < n_fixed) {
     b = idx / fixed_rows;
     const int i = idx - b * fixed_rows;
     r = i < c.n_sys ? i : i + c.k_keep;
     dependent = false;
   } else {
-    idx -= c.batch * fixed_rows;
+    idx -= n_fixed;
     b = idx / c.k_keep;
     r = c.n_sys + (idx - b * c.k_keep);
     dependent = true;
