@@ -57,11 +57,11 @@ typedef enum { VSCAN_SCORE_ROW = 0, VSCAN_SCORE_QK = 1, VSCAN_SCORE_RECEIVED = 2
 typedef enum { VSCAN_SPAN_ONLY = 0, VSCAN_SPAN_FULL = 1 } vscan_softmax_span;
 /* Which unit runs the similarity contraction of vscan_merge. */
 typedef enum {
-  VSCAN_MERGE_AUTO = 0,   /* bf16: INTERLEAVED for kept sets of 129..256, else TENSOR when the shape allows, else SIMT;
-                             f32: SIMT */
+  VSCAN_MERGE_AUTO = 0,   /* bf16: TENSOR when the shape allows, else SIMT; f32: SIMT */
   VSCAN_MERGE_SIMT = 1,   /* fp32 FMA on CUDA cores (the only path for VSCAN_F32) */
-  VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory; group sums in a second
-                             kernel, on the tensor cores too (one-hot matrix products) where the shape allows */
+  VSCAN_MERGE_TENSOR = 2, /* tcgen05 MMA, bf16 inputs, fp32 accumulation in tensor memory (kept sets above 128: the kept
+                             rows are packed first and the MMAs run on CTA pairs); group sums in a second kernel, on
+                             the tensor cores too (one-hot matrix products) where the shape allows */
   VSCAN_MERGE_CLUSTER = 3, /* assignment and group sums in ONE pass over the features: a cluster of dim / 256 CTAs per
                              instance, each owning 256 feature columns, exchanges partial dot products through
                              distributed shared memory (bf16, n_kept <= 64, dim 256 / 512 / 1024, no metric) */

@@ -490,9 +490,10 @@ extern "C" vscan_status vscan_merge(const vscan_merge_desc* d, void* workspace, 
     return launch_merge_cluster(p, stream);
   }
 
-  // assignment and group means in one persistent launch: on request, or by itself where it measured faster
-  // than the two kernels below (kept sets above 128, where those run one or two CTAs per SM)
-  if (d->path == VSCAN_MERGE_INTERLEAVED || (d->path == VSCAN_MERGE_AUTO && d->n_kept > 128)) {
+  // assignment and group means in one persistent launch: on request only.  (It was the choice for kept sets of
+  // 129-256 until the assignment on CTA pairs, which takes packed kept rows at any size above 128: 230 us against
+  // 103 + 79 us for 256 instances with 192 kept tokens.)
+  if (d->path == VSCAN_MERGE_INTERLEAVED) {
     if (merge_interleaved_supported(d->dtype, p)) {
       st = launch_merge_interleaved(p, stream);
       if (st != VSCAN_ERR_UNSUPPORTED || d->path == VSCAN_MERGE_INTERLEAVED) return st;

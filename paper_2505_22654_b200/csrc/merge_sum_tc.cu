@@ -284,6 +284,8 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
   }
 }
 
+// (Kept sets of 129-256 as two halves of 128 slots, 128 columns per item, were measured slower than the CUDA-core
+// group means: 96 against 79 us for 256 instances with 192 kept tokens.)
 static bool plan(const MergeParams& m, Params& p) {
   if (m.dim % 128 != 0 || m.n_kept < 1 || m.n_kept > 128) return false;
   if (m.row_len != m.cls_offset + m.n_tokens) return false;   // rows past the last token must be the copy's zero fill

@@ -930,8 +930,11 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   tc::Params p;
   if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
   // packed kept rows: CTA pairs, each CTA holding half of a stage's kept rows
+  // (kept sets of 129-256 too when the caller asks for the two-kernel path: one round, kept rows packed first)
+  if (!p.b_packed && m.n_kept > 128 && m.kept_packed != nullptr && m.inv_norm != nullptr) { p.b_packed = 1; p.norms_given = 1; }
   const bool pair = p.b_packed && p.norms_given && p.n_pad % 16 == 0;
   if (pair) {
+    while (p.tmem_cols < 2 * p.n_pad) p.tmem_cols *= 2;   // the accumulators alternate between n-chunks of successive items
     p.b_stage_bytes = ((p.n_pad / 2 * tc::kChunkK * 2) + 1023) / 1024 * 1024;
     // (a seventh stage, which just fits, measured slower: 301 us against 294 us at 2048 kept tokens)
     int stages = (215 * 1024) / (p.a_stage_bytes + p.b_stage_bytes);
@@ -954,7 +957,7 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
     const long long items = 1ll * m.instances * pl.splits * pl.ptiles;
     if (items > 0x3fffffffLL) return VSCAN_ERR_UNSUPPORTED;
     pl.items = static_cast<int>(items);
-    const size_t smem = tc::smem_bytes(p);
+    const size_t smem = tc::smem_bytes(p) + (p.n_chunks > 1 ? 0 : static_cast<size_t>(p.n_pad) * sizeof(float));   // two norm buffers
     VSCAN_CUDA_TRY(allow_smem(tc::assign_pair_kernel, smem));
     const int pairs_max = sm_count() / 2;
     const unsigned pairs = static_cast<unsigned>(pl.items < pairs_max ? pl.items : pairs_max);
