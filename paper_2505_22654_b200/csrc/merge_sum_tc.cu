@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kThreads, 1) group_sum_tensor_kernel(const __g
       uint32_t phase = 0;
       const uint32_t base_addr = smem_u32(base), onehot_addr = smem_u32(onehot);
       for (int w = blockIdx.x; w < p.items && ok && !*abort_flag; w += gridDim.x, ++i) {
-        const int b = m.instances - 1 - w / p.slices, col0 = (w - (w / p.slices) * p.slices) * p.m_tiles * 128;
+        const int col0 = (w % p.slices) * p.m_tiles * 128;
         const int my_tiles = min(p.m_tiles, (m.dim - col0) / 128);
         const uint32_t idesc = instr_desc_bf16_bmn(p.n_pad, my_tiles * 128);
         const int acc = i & 1, use = i >> 1;

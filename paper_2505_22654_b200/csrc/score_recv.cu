@@ -20,7 +20,7 @@ namespace recv {
 
 using namespace tc;
 
-constexpr int kThreads = 192;   // warp 0 TMA, warp 1 MMA, warps 2-5 read-back
+constexpr int kThreads = 320;   // warp 0 TMA, warp 1 MMA, warps 2-9 read-back: two warps per quarter of the block rows, 64 columns each
 constexpr int kTile = 128;      // rows of the resident tile (MMA M) and of a streamed tile (MMA N)
 constexpr int kChunkBytes = kTile * 128;   // one [128 rows x 64 elements] box
 
@@ -38,6 +38,7 @@ struct Shared {
   uint64_t tmem_full[2], tmem_empty[2];
   uint32_t tmem_base;
   int abort_flag;
+  float part_a[kTile], part_b[kTile];   // the second column half's (maximum, sum) or column sum of every block row
 };
 
 __device__ __forceinline__ float ex2(float x) {
@@ -67,10 +68,10 @@ __global__ void __launch_bounds__(kThreads) received_kernel(const __grid_constan
 
   if (threadIdx.x == 0) {
     mbar_init(&sh.a_full, 1);
-    // a stage is released by the MMAs that read it (pass 1) or by the four read-back warps, which read its lse2
+    // a stage is released by the MMAs that read it (pass 1) or by the eight read-back warps, which read its lse2
     // values after those MMAs have completed (pass 2)
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], p.pass == 2 ? 4 : 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 4); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], p.pass == 2 ? 8 : 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh.tmem_full[a], 1); mbar_init(&sh.tmem_empty[a], 8); }
     sh.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -125,9 +126,12 @@ __global__ void __launch_bounds__(kThreads) received_kernel(const __grid_constan
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------------------ read-back: one block row per thread
-    const int quarter = warp & 3;
-    const int row = row0 + quarter * 32 + lane;           // query (pass 1) or key (pass 2) of this thread
+    // ------------------------------------------------------------ read-back: one block row and 64 of the block's 128
+    // columns per thread (warps w and w + 4 share a quarter of the rows); the two halves keep their own running
+    // figures and are put together once at the end
+    const int quarter = warp & 3, half = (warp - 2) >> 2;
+    const int r_in = quarter * 32 + lane;                 // row of this thread within the block
+    const int row = row0 + r_in;                          // query (pass 1) or key (pass 2) of this thread
     float run_max = -INFINITY, run_sum = 0.f, col_sum = 0.f;
     bool ok = true;
     for (int t = 0; t < p.tiles; ++t) {
@@ -135,44 +139,46 @@ __global__ void __launch_bounds__(kThreads) received_kernel(const __grid_constan
       if (ok) ok = mbar_wait_warp(&sh.tmem_full[acc], use & 1, abort_flag);
       if (!ok) continue;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTile;
-      const int col0 = t * kTile;
+      const uint32_t taddr = tmem_acc + (static_cast<uint32_t>(quarter * 32) << 16) + acc * kTile + half * 64;
+      const int col0 = t * kTile + half * 64;
       if (p.pass == 1) {
-        // two sweeps over the block row: its maximum first, then the exponentials against the new running maximum
-        float tile_max = -INFINITY;
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
+        // one sweep: per 32 columns the running maximum is raised first, the sum rescaled, the exponentials added
+        for (int c0 = 0; c0 < 64; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(taddr + c0, v);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          float cmax = -INFINITY;
 #pragma unroll
           for (int j = 0; j < 32; ++j)
-            if (col0 + c0 + j < p.n) tile_max = fmaxf(tile_max, __uint_as_float(v[j]) * p.scale_log2e);
-        }
-        const float new_max = fmaxf(run_max, tile_max);
-        float add = 0.f;
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
-          uint32_t v[32];
-          tmem_ld32(taddr + c0, v);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (col0 + c0 + j < p.n) cmax = fmaxf(cmax, __uint_as_float(v[j]) * p.scale_log2e);
+          const float new_max = fmaxf(run_max, cmax);
+          if (new_max > -INFINITY) {
+            float add0 = 0.f, add1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (col0 + c0 + j < p.n) add += ex2(fmaf(__uint_as_float(v[j]), p.scale_log2e, -new_max));
+            for (int j = 0; j < 32; j += 2) {
+              if (col0 + c0 + j < p.n) add0 += ex2(fmaf(__uint_as_float(v[j]), p.scale_log2e, -new_max));
+              if (col0 + c0 + j + 1 < p.n) add1 += ex2(fmaf(__uint_as_float(v[j + 1]), p.scale_log2e, -new_max));
+            }
+            run_sum = run_sum * ex2(run_max - new_max) + (add0 + add1);   // (first columns: 0 * 2^(-inf) = 0)
+            run_max = new_max;
+          }
         }
-        run_sum = run_sum * ex2(run_max - new_max) + add;   // (first tile: 0 * 2^(-inf) = 0)
-        run_max = new_max;
       } else {
         // the copy of the lse2 values completes on the stage's barrier: observe it before reading them
         if (!mbar_wait_warp(&sh.full[s], (t / p.stages) & 1, abort_flag)) { ok = false; continue; }
-        const float* lse = reinterpret_cast<const float*>(lse_ring + s * 512);
-        for (int c0 = 0; c0 < kTile; c0 += 32) {
+        const float* lse = reinterpret_cast<const float*>(lse_ring + s * 512) + half * 64;
+        for (int c0 = 0; c0 < 64; c0 += 32) {
           uint32_t v[32];
           tmem_ld32(taddr + c0, v);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          float add0 = 0.f, add1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int i = col0 + c0 + j;                   // the query of this column
-            if (i < p.n && i != row) col_sum += ex2(fmaf(__uint_as_float(v[j]), p.scale_log2e, -lse[c0 + j]));
+          for (int j = 0; j < 32; j += 2) {
+            const int i0 = col0 + c0 + j;                  // the queries of these two columns
+            if (i0 < p.n && i0 != row) add0 += ex2(fmaf(__uint_as_float(v[j]), p.scale_log2e, -lse[c0 + j]));
+            if (i0 + 1 < p.n && i0 + 1 != row) add1 += ex2(fmaf(__uint_as_float(v[j + 1]), p.scale_log2e, -lse[c0 + j + 1]));
           }
+          col_sum += add0 + add1;
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -182,9 +188,18 @@ __global__ void __launch_bounds__(kThreads) received_kernel(const __grid_constan
         if (p.pass == 2) mbar_arrive(&sh.empty[s]);
       }
     }
-    if (ok && row < p.n) {
-      if (p.pass == 1) p.lse2[static_cast<size_t>(bh) * p.n_pad + row] = run_max + log2f(run_sum);
-      else p.rows[static_cast<size_t>(bh) * p.n + row] = col_sum / static_cast<float>(max(p.n - 1, 1));
+    // ---- the second column half hands its figures to the first, which writes the row's result
+    if (half == 1) { sh.part_a[r_in] = p.pass == 1 ? run_max : col_sum; sh.part_b[r_in] = run_sum; }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (half == 0 && ok && row < p.n) {
+      if (p.pass == 1) {
+        const float m2 = sh.part_a[r_in], s2 = sh.part_b[r_in];
+        const float mx = fmaxf(run_max, m2);
+        const float sum = (run_sum > 0.f ? run_sum * ex2(run_max - mx) : 0.f) + (s2 > 0.f ? s2 * ex2(m2 - mx) : 0.f);
+        p.lse2[static_cast<size_t>(bh) * p.n_pad + row] = mx + log2f(sum);
+      } else {
+        p.rows[static_cast<size_t>(bh) * p.n + row] = (col_sum + sh.part_a[r_in]) / static_cast<float>(max(p.n - 1, 1));
+      }
     }
   }
 
@@ -227,7 +242,9 @@ vscan_status launch_received(const vscan_score_desc* d, void* workspace, float* 
   p.rows = rows_out;
   p.n = d->seq_len; p.n_pad = static_cast<int>(n_pad); p.k_chunks = d->head_dim / 64;
   p.tiles = static_cast<int>(n_pad / kTile);
-  p.stages = p.k_chunks == 1 ? 4 : 3;
+  // two CTAs per SM (shared memory and the 512 columns of tensor memory allow no more): the exponentials of the
+  // read-back, not the loads, bound the kernel (head dim 128: 31 ms with three stages and one CTA per SM, 19 ms with two)
+  p.stages = p.k_chunks == 1 ? 4 : 2;
   p.scale_log2e = d->scale * 1.4426950408889634f;
   CUtensorMap maps[2];
   const void* ptrs[2] = {d->q, d->k};
