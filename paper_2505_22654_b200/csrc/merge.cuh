@@ -14,7 +14,7 @@ struct MergeParams {
   void* merged;         // [instances][n_kept][dim]
   int32_t* counts;      // optional
   void* kept_packed;    // [instances][n_kept rounded up to 256, or to 16 when <= 256][metric_dim] copy of the kept rows   (workspace;
-                        // only for kept sets above 256, where it feeds the tensor path with plain tile loads)
+                        // feeds the tensor paths with plain tile loads: kept sets above 128, and the persistent path)
   int* counters;        // [instances + 1] counters of the persistent path                              (workspace)
   int32_t* order;       // [instances][n_tokens] tokens ordered by slot, long instances only            (workspace)
   int32_t* order_start; // [instances][n_kept + 1] segment starts of `order`                            (workspace)

@@ -276,7 +276,7 @@ __global__ void __launch_bounds__(kThreads) assign_tensor_kernel(const __grid_co
 }
 
 // ---------------------------------------------------------------------------------------------
-// Large kept sets (packed rows, norms from the packing kernel): the assignment on CTA pairs.  A pair of CTAs
+// Kept sets above 128 (packed rows, norms from the packing kernel): the assignment on CTA pairs.  A pair of CTAs
 // (a cluster of two, on the two SMs of one TPC) takes 256 tokens; each CTA loads its own 128 token rows and HALF of
 // the kept rows of a stage, and one MMA of M = 256 issued by the even CTA runs on both SMs, each tensor core reading
 // its own token tile and both halves of the kept rows.  Per 128 tokens and stage an SM takes in 16 KB + n_pad/2 rows
@@ -930,7 +930,8 @@ vscan_status launch_assign_tensor(const MergeParams& m, cudaStream_t stream) {
   tc::Params p;
   if (!tc::plan(m, p)) return VSCAN_ERR_UNSUPPORTED;
   // packed kept rows: CTA pairs, each CTA holding half of a stage's kept rows
-  // (kept sets of 129-256 too when the caller asks for the two-kernel path: one round, kept rows packed first)
+  // kept sets of 129-256 take the same form in one round: with row gathers (48 requests per stage at 192 kept tokens)
+  // the single-CTA kernel is bound by the issue rate of its producer
   if (!p.b_packed && m.n_kept > 128 && m.kept_packed != nullptr && m.inv_norm != nullptr) { p.b_packed = 1; p.norms_given = 1; }
   const bool pair = p.b_packed && p.norms_given && p.n_pad % 16 == 0;
   if (pair) {
